@@ -1,0 +1,206 @@
+"""ctypes front-end of ``conv_oracle.c`` (TEST INFRASTRUCTURE ONLY).
+
+Compiles the C file with gcc on first use (``-O2 -fopenmp``) into
+``oracle/_build/liboracle.so`` and exposes numpy-in / numpy-out functions.
+Argument checking and array allocation only; every sum is formed in the C file.
+"""
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "conv_oracle.c")
+_OUT_DIR = os.path.join(_HERE, "_build")
+_LIB_PATH = os.path.join(_OUT_DIR, "liboracle.so")
+_lock = threading.Lock()
+_lib = None
+
+_c_ll = ctypes.c_longlong
+_c_int = ctypes.c_int
+_vp = ctypes.c_void_p
+
+
+def build_oracle(force: bool = False) -> str:
+    """Compile the C oracle if the shared object is missing or stale."""
+    os.makedirs(_OUT_DIR, exist_ok=True)
+    stale = (not os.path.exists(_LIB_PATH)
+             or os.path.getmtime(_LIB_PATH) < os.path.getmtime(_SRC))
+    if force or stale:
+        tmp = _LIB_PATH + ".tmp.%d" % os.getpid()
+        cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11",
+               "-o", tmp, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+        os.replace(tmp, _LIB_PATH)
+    return _LIB_PATH
+
+
+def _load():
+    global _lib
+    with _lock:
+        if _lib is None:
+            lib = ctypes.CDLL(build_oracle())
+            lib.oracle_num_threads.restype = _c_int
+            lib.oracle_set_num_threads.argtypes = [_c_int]
+            lib.oracle_conv1d_f32.argtypes = [_vp, _c_ll, _vp, _c_int, _vp, _vp]
+            lib.oracle_conv1d_f32_taps_outer.argtypes = [_vp, _c_ll, _vp, _c_int, _vp]
+            lib.oracle_conv1d_f32_at.argtypes = [_vp, _c_ll, _vp, _c_int, _vp, _c_ll, _vp, _vp]
+            lib.oracle_conv2d_f32.argtypes = [_vp, _c_int, _c_int, _c_ll, _vp, _c_int, _c_int,
+                                              _vp, _vp, _c_ll]
+            lib.oracle_conv2d_f32_taps_outer.argtypes = [_vp, _c_int, _c_int, _c_ll, _vp, _c_int,
+                                                         _c_int, _vp, _c_ll]
+            lib.oracle_conv2d_f32_at.argtypes = [_vp, _c_int, _c_int, _c_ll, _vp, _c_int, _c_int,
+                                                 _vp, _vp, _c_ll, _vp, _vp]
+            lib.oracle_conv1d_u8s8_s32.argtypes = [_vp, _c_ll, _vp, _c_int, _vp]
+            lib.oracle_conv2d_u8s8_s32.argtypes = [_vp, _c_int, _c_int, _c_ll, _vp, _c_int, _c_int,
+                                                   _vp, _c_ll]
+            lib.oracle_conv2d_u8s8_i64.argtypes = [_vp, _c_int, _c_int, _c_ll, _vp, _c_int, _c_int,
+                                                   _vp, _c_ll]
+            for name in ("oracle_set_num_threads", "oracle_conv1d_f32",
+                         "oracle_conv1d_f32_taps_outer", "oracle_conv1d_f32_at",
+                         "oracle_conv2d_f32", "oracle_conv2d_f32_taps_outer",
+                         "oracle_conv2d_f32_at", "oracle_conv1d_u8s8_s32",
+                         "oracle_conv2d_u8s8_s32", "oracle_conv2d_u8s8_i64"):
+                getattr(lib, name).restype = None
+            _lib = lib
+    return _lib
+
+
+def _ptr(a: np.ndarray):
+    return a.ctypes.data_as(_vp)
+
+
+def _as(a, dtype, ndim):
+    a = np.ascontiguousarray(a, dtype=dtype)
+    if a.ndim != ndim:
+        raise ValueError("expected %d-D array, got %d-D" % (ndim, a.ndim))
+    return a
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def set_num_threads(n: int) -> None:
+    _load().oracle_set_num_threads(int(n))
+
+
+def conv1d_f32(x, w, want_scale=True):
+    """Eq. 2 in fp64. Returns (y, S) with S = sum |w||x| per output (or None)."""
+    x = _as(x, np.float32, 1)
+    w = _as(w, np.float32, 1)
+    n, q = x.shape[0], w.shape[0]
+    if q < 1 or n < q:
+        raise ValueError("need 1 <= Q <= N")
+    y = np.empty(n - q + 1, dtype=np.float64)
+    s = np.empty(n - q + 1, dtype=np.float64) if want_scale else None
+    _load().oracle_conv1d_f32(_ptr(x), n, _ptr(w), q, _ptr(y), _ptr(s) if want_scale else None)
+    return y, s
+
+
+def conv1d_f32_taps_outer(x, w):
+    x = _as(x, np.float32, 1)
+    w = _as(w, np.float32, 1)
+    n, q = x.shape[0], w.shape[0]
+    if q < 1 or n < q:
+        raise ValueError("need 1 <= Q <= N")
+    y = np.empty(n - q + 1, dtype=np.float64)
+    _load().oracle_conv1d_f32_taps_outer(_ptr(x), n, _ptr(w), q, _ptr(y))
+    return y
+
+
+def conv1d_f32_at(x, w, pos):
+    """Eq. 2 at the output positions ``pos`` only. Returns (y, S)."""
+    x = _as(x, np.float32, 1)
+    w = _as(w, np.float32, 1)
+    pos = _as(pos, np.int64, 1)
+    n, q = x.shape[0], w.shape[0]
+    if pos.size and (pos.min() < 0 or pos.max() > n - q):
+        raise ValueError("position outside the valid output range")
+    y = np.empty(pos.size, dtype=np.float64)
+    s = np.empty(pos.size, dtype=np.float64)
+    _load().oracle_conv1d_f32_at(_ptr(x), n, _ptr(w), q, _ptr(pos), pos.size, _ptr(y), _ptr(s))
+    return y, s
+
+
+def conv2d_f32(x, w, want_scale=True):
+    """Eq. 3 in fp64 on one image x[H][W] with filter w[P][Q]. Returns (y, S)."""
+    x = _as(x, np.float32, 2)
+    w = _as(w, np.float32, 2)
+    h, wd = x.shape
+    p, q = w.shape
+    if p < 1 or q < 1 or h < p or wd < q:
+        raise ValueError("filter larger than image")
+    y = np.empty((h - p + 1, wd - q + 1), dtype=np.float64)
+    s = np.empty_like(y) if want_scale else None
+    _load().oracle_conv2d_f32(_ptr(x), wd, h, wd, _ptr(w), q, p, _ptr(y),
+                              _ptr(s) if want_scale else None, wd - q + 1)
+    return y, s
+
+
+def conv2d_f32_taps_outer(x, w):
+    x = _as(x, np.float32, 2)
+    w = _as(w, np.float32, 2)
+    h, wd = x.shape
+    p, q = w.shape
+    if p < 1 or q < 1 or h < p or wd < q:
+        raise ValueError("filter larger than image")
+    y = np.empty((h - p + 1, wd - q + 1), dtype=np.float64)
+    _load().oracle_conv2d_f32_taps_outer(_ptr(x), wd, h, wd, _ptr(w), q, p, _ptr(y), wd - q + 1)
+    return y
+
+
+def conv2d_f32_at(x, w, rows, cols):
+    """Eq. 3 at output positions (rows[i], cols[i]) only. Returns (y, S)."""
+    x = _as(x, np.float32, 2)
+    w = _as(w, np.float32, 2)
+    rows = _as(rows, np.int64, 1)
+    cols = _as(cols, np.int64, 1)
+    h, wd = x.shape
+    p, q = w.shape
+    if rows.shape != cols.shape:
+        raise ValueError("rows and cols differ in length")
+    if rows.size and (rows.min() < 0 or rows.max() > h - p or cols.min() < 0 or cols.max() > wd - q):
+        raise ValueError("position outside the valid output range")
+    y = np.empty(rows.size, dtype=np.float64)
+    s = np.empty(rows.size, dtype=np.float64)
+    _load().oracle_conv2d_f32_at(_ptr(x), wd, h, wd, _ptr(w), q, p, _ptr(rows), _ptr(cols),
+                                 rows.size, _ptr(y), _ptr(s))
+    return y, s
+
+
+def conv1d_u8s8_s32(x, w):
+    x = _as(x, np.uint8, 1)
+    w = _as(w, np.int8, 1)
+    n, q = x.shape[0], w.shape[0]
+    if q < 1 or n < q:
+        raise ValueError("need 1 <= Q <= N")
+    y = np.empty(n - q + 1, dtype=np.int32)
+    _load().oracle_conv1d_u8s8_s32(_ptr(x), n, _ptr(w), q, _ptr(y))
+    return y
+
+
+def conv2d_u8s8_s32(x, w):
+    x = _as(x, np.uint8, 2)
+    w = _as(w, np.int8, 2)
+    h, wd = x.shape
+    p, q = w.shape
+    if p < 1 or q < 1 or h < p or wd < q:
+        raise ValueError("filter larger than image")
+    y = np.empty((h - p + 1, wd - q + 1), dtype=np.int32)
+    _load().oracle_conv2d_u8s8_s32(_ptr(x), wd, h, wd, _ptr(w), q, p, _ptr(y), wd - q + 1)
+    return y
+
+
+def conv2d_u8s8_i64(x, w):
+    x = _as(x, np.uint8, 2)
+    w = _as(w, np.int8, 2)
+    h, wd = x.shape
+    p, q = w.shape
+    if p < 1 or q < 1 or h < p or wd < q:
+        raise ValueError("filter larger than image")
+    y = np.empty((h - p + 1, wd - q + 1), dtype=np.int64)
+    _load().oracle_conv2d_u8s8_i64(_ptr(x), wd, h, wd, _ptr(w), q, p, _ptr(y), wd - q + 1)
+    return y
