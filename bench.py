@@ -1,0 +1,500 @@
+#!/usr/bin/env python
+"""Benchmark of the warp-systolic convolution library on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload cfgN]
+
+Prints ONE JSON line.  A "step" is one pass of the whole hot path over the
+workload: every filter size of the configuration through every systolic design
+(weight-, output-, input-stationary), one kernel launch each.  The default
+workload is configuration 2 (1-D fp32, N = 2^26, Q in {4, 16, 32}: nine
+launches per step); the metric is output elements per second.
+
+* value      device-resident inputs, CUDA-event time around K steps
+* e2e        the same step through the host-buffer C-ABI entry points (pinned
+             host memory, host<->device copies inside the timed region)
+* roofline   the kernel with the largest share of the step, algorithmic bytes /
+             its average launch time (per-launch CUDA events) vs the measured
+             HBM copy bandwidth of this machine (MEASURED_PEAKS.json)
+* cpu_baseline  the CPU oracle timed on this machine's cores on a bounded sample
+* detail     per (configuration, filter, design): time, Gpix/s, GB/s, roofline
+             fraction (all five configurations unless --no-detail)
+
+--impl reference times the CPU oracle (the only reference there is: the paper
+ships no code and its comparison system is Intel fixed-function hardware).
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+HBM_FALLBACK_GBS = 6650.0
+SM_COUNT = 148
+FP32_LANES_PER_SM = 128
+NAMES = {0: "WS", 1: "OS", 2: "IS"}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured", float(d.get("sm_max_mhz", 1965.0))
+    except Exception:
+        return HBM_FALLBACK_GBS, "fallback", 1965.0
+
+
+# --------------------------------------------------------------------------- clocks
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc, self.thread = index, [], None, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, pw, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1])); pw.append(float(r[2]))
+            except ValueError:
+                continue
+            for name, flag in zip(names, r[3:7]):
+                if flag.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------- workloads
+
+
+class Case:
+    """One kernel launch of a workload: a (filter, design) pair on resident device buffers."""
+
+    def __init__(self, cfg, label, design, launch, n_out, alg_bytes, macs):
+        self.cfg, self.label, self.design, self.launch = cfg, label, design, launch
+        self.n_out, self.alg_bytes, self.macs = n_out, alg_bytes, macs
+        self.times_ms = []
+
+
+def build_cases(cfg_id, device, designs=(0, 1, 2), scale=None):
+    """Generate the configuration's inputs, copy them to the device, return (cases, keepalive)."""
+    import torch
+    from paper_2010_15884_b200 import binding as B
+    from paper_2010_15884_b200 import inputs
+    x, ws = inputs.make_config(cfg_id, scale)
+    xd = torch.from_numpy(x).to(device)
+    cases, keep = [], [xd]
+    kind = inputs.CONFIGS[cfg_id]["kind"]
+    stream = torch.cuda.current_stream().cuda_stream
+    dtype = B.U8S8_S32 if kind == "2d_u8s8" else B.F32
+
+    def checked(call, *cargs):
+        def run():
+            st = call(*cargs)
+            if st != 0:
+                raise B.SysconvError(st, call.__name__)
+        return run
+
+    for key, w in ws.items():
+        w = np.ascontiguousarray(w)
+        keep.append(w)
+        if kind == "1d_f32":
+            q = key
+            n = x.shape[0]
+            n_out = n - q + 1
+            yd = torch.empty(n_out, dtype=torch.float32, device=device)
+            alg = 4 * n + 4 * n_out
+            macs = n_out * q
+            label = "Q=%d" % q
+            mk = (lambda d, w=w, yd=yd, q=q, n=n, n_out=n_out:
+                  checked(B.sysconv1d, xd.data_ptr(), n, n, w, q, yd.data_ptr(), n_out, 1, dtype, d, stream))
+        else:
+            p, q = key
+            batch, h, wd = x.shape
+            oh, ow = h - p + 1, wd - q + 1
+            # output rows padded to a 16-byte multiple so that every row starts aligned
+            y_pitch = (ow + 3) // 4 * 4
+            yd = torch.empty((batch, oh, y_pitch), dtype=torch.float32 if kind == "2d_f32" else torch.int32,
+                             device=device)
+            n_out = batch * oh * ow
+            alg = x.size * x.itemsize + 4 * n_out
+            macs = n_out * p * q
+            label = "%dx%d" % (p, q)
+            mk = (lambda d, w=w, yd=yd, p=p, q=q, h=h, wd=wd, oh=oh, y_pitch=y_pitch, batch=batch:
+                  checked(B.sysconv2d, xd.data_ptr(), wd, h, wd, h * wd, w, q, p, yd.data_ptr(), y_pitch,
+                          oh * y_pitch, batch, dtype, d, stream))
+        keep.append(yd)
+        for d in designs:
+            cases.append(Case(cfg_id, label, d, mk(d), n_out, alg, macs))
+    return cases, keep
+
+
+def roofline_time_s(case, hbm_gbs, sm_mhz):
+    """max(bytes / HBM bandwidth, MACs / plain-ALU MAC rate) for one launch."""
+    t_mem = case.alg_bytes / (hbm_gbs * 1e9)
+    mac_rate = SM_COUNT * FP32_LANES_PER_SM * sm_mhz * 1e6
+    t_alu = case.macs / mac_rate
+    return max(t_mem, t_alu), ("hbm" if t_mem >= t_alu else "alu")
+
+
+def time_cases_individually(cases, warmup, reps, flush):
+    """Per-launch CUDA-event timing, each launch bracketed by its own event pair."""
+    import torch
+    for c in cases:
+        for _ in range(warmup):
+            c.launch()
+    torch.cuda.synchronize()
+    for c in cases:
+        c.times_ms = []
+        for _ in range(reps):
+            if flush is not None:
+                flush.add_(1.0)          # > L2 write between iterations
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            c.launch()
+            e1.record()
+            e1.synchronize()
+            c.times_ms.append(e0.elapsed_time(e1))
+
+
+def detail_rows(cases, hbm_gbs, peak_kind, sm_max):
+    rows = []
+    for c in cases:
+        med = statistics.median(c.times_ms)
+        t_roof, bound = roofline_time_s(c, hbm_gbs, sm_max)
+        rows.append({
+            "config": c.cfg, "filter": c.label, "design": NAMES[c.design],
+            "ms_median": round(med, 5), "ms_min": round(min(c.times_ms), 5),
+            "gpix_s": round(c.n_out / (med * 1e-3) / 1e9, 3),
+            "gb_s": round(c.alg_bytes / (med * 1e-3) / 1e9, 1),
+            "roofline_bound": bound,
+            "roofline_frac": round(t_roof / (med * 1e-3), 4),
+            "hbm_frac": round(c.alg_bytes / (med * 1e-3) / 1e9 / hbm_gbs, 4),
+        })
+    return rows
+
+
+# --------------------------------------------------------------------------- CPU oracle arm
+
+
+def oracle_sample(cfg_id):
+    """Time the oracle, as it stands, on a bounded sample of the configuration.
+
+    Returns (outputs, seconds, threads, description).  1-D: one pass per filter length over the first
+    2^24 samples.  2-D: one pass per filter size over the first 1024 rows of image 0.
+    """
+    import oracle
+    from paper_2010_15884_b200 import inputs
+    x, ws = inputs.make_config(cfg_id)
+    kind = inputs.CONFIGS[cfg_id]["kind"]
+    outs = 0
+    if kind == "1d_f32":
+        x = x[: 1 << 24]
+        oracle.conv1d_f32(x[: 1 << 16], next(iter(ws.values())), want_scale=False)   # load + warm
+        t0 = time.perf_counter()
+        for w in ws.values():
+            outs += oracle.conv1d_f32(x, w, want_scale=False)[0].size
+        what = "one fp64 pass of Eq. 2 per filter length over the first %d samples" % x.shape[0]
+    else:
+        img = np.ascontiguousarray(x[0][:1024])
+        f = oracle.conv2d_f32 if kind == "2d_f32" else (lambda a, b, want_scale=False: (oracle.conv2d_u8s8_s32(a, b), None))
+        f(img[:32], next(iter(ws.values())), want_scale=False)
+        t0 = time.perf_counter()
+        for w in ws.values():
+            outs += f(img, w, want_scale=False)[0].size
+        what = "one pass of Eq. 3 per filter size over the first %d rows of image 0" % img.shape[0]
+    return outs, time.perf_counter() - t0, oracle.num_threads(), what
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle on the host cores, rank 0 only."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    sample_n = 1 << 24
+    import oracle
+    from paper_2010_15884_b200 import inputs
+    x, ws = inputs.make_config(2)
+    x = x[:sample_n]
+    for _ in range(max(args.warmup, 1)):
+        oracle.conv1d_f32(x[: 1 << 18], ws[4], want_scale=False)
+    outs, t0 = 0, time.perf_counter()
+    for _ in range(args.steps):
+        for q, w in ws.items():
+            y, _ = oracle.conv1d_f32(x, w, want_scale=False)
+            outs += 3 * y.size                          # the three designs share this one definition
+    dt = time.perf_counter() - t0
+    value = outs / dt / 1e9
+    sample = ("per step: one fp64 pass of Eq. 2 per filter length (4, 16, 32) over the first 2^24 samples of "
+              "configuration 2, counted once per design")
+    line = {
+        "impl": "reference", "metric": "output elements/s", "value": round(value, 4), "unit": "Gpix/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": round(dt / args.steps * 1e3, 3), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "cfg2: 1-D fp32 N=2^26, Q in {4,16,32}, designs WS/OS/IS", "sample": sample},
+        "cpu_baseline": {"value": round(value, 4), "unit": "Gpix/s", "cores": oracle.num_threads(),
+                         "kind": "oracle", "sample": sample},
+        "e2e": {"value": round(value, 4), "unit": "Gpix/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- our arm
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2010_15884_b200 import binding as B
+    from paper_2010_15884_b200 import inputs, shard
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=device)
+    B.load_library()
+    hbm_gbs, peak_kind, sm_max = measured_peaks()
+
+    cfg_id = int(args.workload.replace("cfg", ""))
+    cases, keep = build_cases(cfg_id, device)          # every rank holds its own copy: weak scaling
+    outputs_per_step = sum(c.n_out for c in cases)
+
+    # ---- device-resident timing: W warm-up steps, then exactly K timed steps
+    small = max(c.alg_bytes for c in cases) < 256e6     # fits L2: flush between steps
+    flush = torch.zeros(64 << 20, dtype=torch.float32, device=device) if small else None
+    for _ in range(args.warmup):
+        for c in cases:
+            c.launch()
+    launches0 = B.launch_count()
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    torch.cuda.synchronize()
+    shard.barrier(world)
+    ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in cases]
+          for _ in range(args.steps)]
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    flush_ms = 0.0
+    start.record()
+    for k in range(args.steps):
+        if flush is not None:
+            f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            f0.record(); flush.add_(1.0); f1.record()
+            ev[k].append((f0, f1))
+        for i, c in enumerate(cases):
+            ev[k][i][0].record()
+            c.launch()
+            ev[k][i][1].record()
+    stop.record()
+    torch.cuda.synchronize()
+    shard.barrier(world)
+    clocks = sampler.stop() if rank == 0 else None
+    launches = B.launch_count() - launches0
+    total_ms = start.elapsed_time(stop)
+    if flush is not None:
+        flush_ms = sum(ev[k][-1][0].elapsed_time(ev[k][-1][1]) for k in range(args.steps))
+        total_ms -= flush_ms
+    for i, c in enumerate(cases):
+        c.times_ms = [ev[k][i][0].elapsed_time(ev[k][i][1]) for k in range(args.steps)]
+    total_ms = shard.max_over_ranks(total_ms, world, device)
+    value = world * outputs_per_step * args.steps / (total_ms * 1e-3) / 1e9
+
+    # ---- roofline of the kernel with the largest share of the step
+    top = max(cases, key=lambda c: sum(c.times_ms))
+    avg_s = statistics.mean(top.times_ms) * 1e-3
+    t_roof, bound = roofline_time_s(top, hbm_gbs, sm_max)
+    roofline = {
+        "kernel": "%s %s" % (NAMES[top.design], top.label), "bound": "hbm",
+        "achieved": round(top.alg_bytes / avg_s / 1e9, 1), "peak": hbm_gbs, "unit": "GB/s",
+        "frac": round(top.alg_bytes / avg_s / 1e9 / hbm_gbs, 4), "peak_source": "of " + peak_kind,
+        "traffic": ncu_traffic(cfg_id, top),
+        "share_of_step": round(sum(top.times_ms) / sum(sum(c.times_ms) for c in cases), 4),
+        "alu_time_frac": round(top.macs / (SM_COUNT * FP32_LANES_PER_SM * sm_max * 1e6) / avg_s, 4),
+    }
+
+    # ---- end to end through the host-buffer entry points (rank-local pinned buffers)
+    e2e = run_e2e(cfg_id, device, args, world)
+
+    line = {
+        "metric": "output elements/s", "value": round(value, 3), "unit": "Gpix/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(total_ms / args.steps, 4),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32" if inputs.CONFIGS[cfg_id]["kind"] != "2d_u8s8" else "s32", "data": "synthetic",
+        "config": {"workload": "cfg%d: %s; every filter x designs WS/OS/IS, one launch each"
+                               % (cfg_id, inputs.CONFIGS[cfg_id]["note"]),
+                   "launches_per_step": len(cases),
+                   "l2": "flushed between steps (128 MiB write, excluded from the time)" if small
+                         else "inputs larger than L2 (268 MB signal per launch)",
+                   "per_rank": "each rank convolves its own copy (independent problems, no collective)"},
+        "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+    }
+    if rank == 0:
+        outs, secs, cores, what = oracle_sample(cfg_id)
+        line["cpu_baseline"] = {
+            "value": round(outs / secs / 1e9, 4), "unit": "Gpix/s", "cores": cores, "kind": "oracle",
+            "sample": "%s of configuration %d (%.1f s)" % (what, cfg_id, secs)}
+        line["per_kernel"] = detail_rows(cases, hbm_gbs, peak_kind, sm_max)
+        if not args.no_detail and world == 1:
+            del cases, keep
+            torch.cuda.empty_cache()
+            line["detail"] = all_config_detail(device, hbm_gbs, peak_kind, sm_max, skip=cfg_id,
+                                               reps=args.detail_reps)
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+_NCU_TRAFFIC = None
+
+
+def ncu_traffic(cfg_id, case):
+    """DRAM bytes per launch of this kernel from the committed ncu summary, if one covers it."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        with open(path) as f:
+            table = json.load(f)
+        return table.get("cfg%d %s %s" % (cfg_id, NAMES[case.design], case.label))
+    except Exception:
+        return None
+
+
+def run_e2e(cfg_id, device, args, world):
+    """The same step from pinned HOST buffers through sysconv*_host (copies inside the timed region)."""
+    import torch
+    from paper_2010_15884_b200 import binding as B
+    from paper_2010_15884_b200 import inputs, shard
+    x, ws = inputs.make_config(cfg_id)
+    kind = inputs.CONFIGS[cfg_id]["kind"]
+    dtype = B.U8S8_S32 if kind == "2d_u8s8" else B.F32
+    xh = torch.from_numpy(x).pin_memory()
+    jobs, h2d, d2h, outputs = [], 0, 0, 0
+    for key, w in ws.items():
+        if kind == "1d_f32":
+            yh = torch.empty(x.shape[0] - key + 1, dtype=torch.float32).pin_memory()
+            wbytes = B.host_workspace_bytes(tuple(x.shape), (key,), dtype)
+            call = B.sysconv1d_host
+        else:
+            p, q = key
+            yh = torch.empty((x.shape[0], x.shape[1] - p + 1, x.shape[2] - q + 1),
+                             dtype=torch.int32 if dtype == B.U8S8_S32 else torch.float32).pin_memory()
+            wbytes = B.host_workspace_bytes(tuple(x.shape), (p, q), dtype)
+            call = B.sysconv2d_host
+        for d in (0, 1, 2):
+            jobs.append((call, w, yh, d))
+            h2d += xh.numel() * xh.element_size()
+            d2h += yh.numel() * yh.element_size()
+            outputs += yh.numel()
+    work = torch.empty(max(B.host_workspace_bytes(tuple(x.shape), ((k,) if kind == "1d_f32" else k), dtype)
+                           for k in ws), dtype=torch.uint8, device=device)
+    steps = max(1, min(args.steps, args.e2e_steps))
+
+    def one_step():
+        for call, w, yh, d in jobs:
+            if call is B.sysconv1d_host:
+                call(xh, w, yh, d, work)
+            else:
+                call(xh, w, yh, d, work, dtype=dtype)
+
+    one_step()
+    torch.cuda.synchronize()
+    shard.barrier(world)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        one_step()
+    e1.record()
+    torch.cuda.synchronize()
+    shard.barrier(world)
+    ms = shard.max_over_ranks(e0.elapsed_time(e1), world, device)
+    return {"value": round(world * outputs * steps / (ms * 1e-3) / 1e9, 4), "unit": "Gpix/s",
+            "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": steps,
+            "ms_per_step": round(ms / steps, 3),
+            "path": "sysconv1d_host/sysconv2d_host: pinned host -> device workspace -> kernel -> pinned host"}
+
+
+def all_config_detail(device, hbm_gbs, peak_kind, sm_max, skip, reps):
+    import torch
+    rows = []
+    flush = torch.zeros(64 << 20, dtype=torch.float32, device=device)
+    for cfg_id in (1, 3, 4, 5):
+        if cfg_id == skip:
+            continue
+        cases, keep = build_cases(cfg_id, device)
+        small = max(c.alg_bytes for c in cases) < 256e6
+        time_cases_individually(cases, 3, reps, flush if small else None)
+        rows += detail_rows(cases, hbm_gbs, peak_kind, sm_max)
+        del cases, keep
+        torch.cuda.empty_cache()
+    return rows
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
+    ap.add_argument("--no-detail", action="store_true", help="skip the per-kernel table of the other configurations")
+    ap.add_argument("--detail-reps", type=int, default=10)
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

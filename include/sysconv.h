@@ -1,0 +1,136 @@
+/*
+ * sysconv -- 1-D and 2-D valid-mode convolution executed as linear software
+ * systolic arrays on the lanes of a warp (NVIDIA B200, sm_100a).
+ *
+ * C ABI of libsysconv.so.  Plain pointers and sizes only.
+ *
+ * The operation (correlation form, no filter flip, valid mode only):
+ *
+ *   1-D, Eq. 2 of the paper:   y[c]    = sum_{k<Q}           w[k]    * x[c + k],       c in [0, N-Q]
+ *   2-D, Eq. 3 of the paper:   y[r][c] = sum_{p<P} sum_{q<Q} w[p][q] * x[r+p][c+q],
+ *                              r in [0, H-P], c in [0, W-Q]
+ *
+ * Each call picks one of the paper's systolic designs (Section 3.1, Table 2,
+ * Section 5); all designs produce the same sums, they differ in which operand
+ * stays in a processing element and which one moves between neighbours:
+ *
+ *   SYSCONV_WS  weight-stationary  = BSM: inputs broadcast, weights stay, partial sums migrate
+ *   SYSCONV_OS  output-stationary  = FBS: inputs forwarded, weights broadcast, partial sums stay
+ *   SYSCONV_IS  input-stationary   = SBM: inputs stay, weights broadcast, partial sums migrate
+ *
+ * (The paper gives SBM and FBS in 2-D; the 2-D weight-stationary design is this
+ * library's own extension of BSM: PE q keeps filter column q.)
+ *
+ * Data types:
+ *   SYSCONV_F32       x, w, y are float; fp32 fused multiply-add accumulation
+ *   SYSCONV_U8S8_S32  x is uint8 (zero-extended), w is int8 (sign-extended),
+ *                     y is int32 with exact int32 accumulation
+ *
+ * Conventions common to every entry point
+ *   - Layout: row-major, the column index c is contiguous; pitches and batch
+ *     strides are in ELEMENTS of the respective array (not bytes).
+ *   - The filter pointer is HOST memory: w[k] in 1-D, w[p*Q + q] in 2-D.  It is
+ *     copied by value into the launch, so it may be freed or changed as soon as
+ *     the call returns.
+ *   - Ownership: the caller owns every buffer.  The library allocates no
+ *     device memory and keeps no state between calls except a launch counter.
+ *   - Asynchrony: the work is enqueued on `stream` (a cudaStream_t passed as
+ *     void*, NULL = the default stream); the call does not synchronise.
+ *   - x and y must not overlap.
+ *   - Supported sizes: 1-D: 1 <= Q <= 32.  2-D: 1 <= P <= 15 and 1 <= Q <= 15.
+ *     Any N, W, H, batch >= 1 that fit the index types; any pitch >= row length.
+ *     Pointers need only be aligned to their element type (16-byte aligned
+ *     rows run faster).
+ *   - Errors: every function returns a sysconv_status; nothing throws, aborts
+ *     or traps.  SYSCONV_EINVAL: null pointer, non-positive size, filter larger
+ *     than the input, pitch/stride smaller than the row/array, unknown enum.
+ *     SYSCONV_EUNSUPPORTED: filter size outside the compiled range.
+ *     SYSCONV_ECUDA: the CUDA runtime reported an error at launch.
+ */
+#ifndef SYSCONV_H_
+#define SYSCONV_H_
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SYSCONV_OK = 0,
+    SYSCONV_EINVAL = 1,
+    SYSCONV_EUNSUPPORTED = 2,
+    SYSCONV_ECUDA = 3,
+    SYSCONV_ETIMEOUT = 4
+} sysconv_status;
+
+typedef enum {
+    SYSCONV_WS = 0, /* BSM */
+    SYSCONV_OS = 1, /* FBS */
+    SYSCONV_IS = 2  /* SBM */
+} sysconv_design;
+
+typedef enum {
+    SYSCONV_F32 = 0,
+    SYSCONV_U8S8_S32 = 1
+} sysconv_dtype;
+
+/*
+ * 1-D convolution, Eq. 2.  `batch` independent signals share one filter:
+ * signal b starts at x_dev + b*x_batch_stride and holds n elements; its n-q+1
+ * outputs go to y_dev + b*y_batch_stride.
+ *   x_dev, y_dev   DEVICE pointers (float/float or uint8/int32 by dtype)
+ *   w_host         HOST pointer to q taps (float or int8 by dtype)
+ *   strides        in elements; ignored when batch == 1 (pass 0 or anything)
+ */
+int sysconv1d(const void *x_dev, long long n, long long x_batch_stride,
+              const void *w_host, int q,
+              void *y_dev, long long y_batch_stride, int batch,
+              int dtype, int design, void *stream);
+
+/*
+ * 2-D convolution, Eq. 3.  Image b starts at x_dev + b*x_batch_stride, has
+ * `height` rows of `width` elements, rows x_pitch elements apart.  The
+ * (height-p+1) x (width-q+1) outputs of image b go to y_dev + b*y_batch_stride,
+ * rows y_pitch elements apart.  `q` is the filter WIDTH (pairs with columns),
+ * `p` the filter HEIGHT; w_host holds p*q taps, w[pp*q + qq].
+ */
+int sysconv2d(const void *x_dev, int width, int height, long long x_pitch, long long x_batch_stride,
+              const void *w_host, int q, int p,
+              void *y_dev, long long y_pitch, long long y_batch_stride, int batch,
+              int dtype, int design, void *stream);
+
+/*
+ * The same two operations for callers whose data lives in HOST memory
+ * (densely packed: pitch = row length, batch stride = array size).  The call
+ * enqueues, on `stream`: the host-to-device copy of x into the caller's device
+ * workspace, the kernel, and the device-to-host copy of y; it does not
+ * synchronise (synchronise the stream before reading y_host).  Copies overlap
+ * only if the host buffers are page-locked.
+ *   workspace_dev / workspace_bytes   DEVICE scratch owned by the caller, at
+ *       least sysconv*_host_workspace_bytes(...) bytes, 256-byte aligned.
+ * Returns SYSCONV_EINVAL if the workspace is too small.
+ */
+long long sysconv1d_host_workspace_bytes(long long n, int q, int batch, int dtype);
+long long sysconv2d_host_workspace_bytes(int width, int height, int q, int p, int batch, int dtype);
+
+int sysconv1d_host(const void *x_host, long long n, const void *w_host, int q,
+                   void *y_host, int batch, int dtype, int design,
+                   void *workspace_dev, long long workspace_bytes, void *stream);
+
+int sysconv2d_host(const void *x_host, int width, int height, const void *w_host, int q, int p,
+                   void *y_host, int batch, int dtype, int design,
+                   void *workspace_dev, long long workspace_bytes, void *stream);
+
+/* Text for a sysconv_status / sysconv_design value ("?" if unknown). Static storage. */
+const char *sysconv_status_string(int status);
+const char *sysconv_design_name(int design);
+
+/* Library version, major*10000 + minor*100 + patch. */
+int sysconv_version(void);
+
+/* Number of kernels this library has launched in this process so far. */
+long long sysconv_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SYSCONV_H_ */

@@ -1,0 +1,230 @@
+"""Thin ctypes binding of libsysconv.so (see include/sysconv.h).
+
+Argument marshalling only: every step of the computation runs in the CUDA
+library.  There is no CPU fallback; if the library cannot be loaded every call
+raises.  PyTorch is used for device memory and streams.
+"""
+import ctypes
+import os
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_NAME = "libsysconv.so"
+
+WS, OS, IS = 0, 1, 2
+F32, U8S8_S32 = 0, 1
+DESIGN_NAMES = {WS: "WS", OS: "OS", IS: "IS"}
+_DESIGN_BY_NAME = {"WS": WS, "BSM": WS, "OS": OS, "FBS": OS, "IS": IS, "SBM": IS}
+
+_c_ll = ctypes.c_longlong
+_c_int = ctypes.c_int
+_vp = ctypes.c_void_p
+
+_lib = None
+
+
+class SysconvError(RuntimeError):
+    def __init__(self, status, where):
+        self.status = int(status)
+        super().__init__("%s failed: status %d (%s)" % (where, status, status_string(status)))
+
+
+def library_path():
+    return os.path.join(_HERE, _LIB_NAME)
+
+
+def load_library():
+    """Load libsysconv.so (built in-tree by paper_2010_15884_b200.build). Raises if missing."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = library_path()
+    if not os.path.exists(path):
+        raise SysconvError(-1, "loading %s (not built: run python -m paper_2010_15884_b200.build)" % path)
+    lib = ctypes.CDLL(path)
+    lib.sysconv1d.restype = _c_int
+    lib.sysconv1d.argtypes = [_vp, _c_ll, _c_ll, _vp, _c_int, _vp, _c_ll, _c_int, _c_int, _c_int, _vp]
+    lib.sysconv2d.restype = _c_int
+    lib.sysconv2d.argtypes = [_vp, _c_int, _c_int, _c_ll, _c_ll, _vp, _c_int, _c_int, _vp, _c_ll, _c_ll,
+                              _c_int, _c_int, _c_int, _vp]
+    lib.sysconv1d_host_workspace_bytes.restype = _c_ll
+    lib.sysconv1d_host_workspace_bytes.argtypes = [_c_ll, _c_int, _c_int, _c_int]
+    lib.sysconv2d_host_workspace_bytes.restype = _c_ll
+    lib.sysconv2d_host_workspace_bytes.argtypes = [_c_int, _c_int, _c_int, _c_int, _c_int, _c_int]
+    lib.sysconv1d_host.restype = _c_int
+    lib.sysconv1d_host.argtypes = [_vp, _c_ll, _vp, _c_int, _vp, _c_int, _c_int, _c_int, _vp, _c_ll, _vp]
+    lib.sysconv2d_host.restype = _c_int
+    lib.sysconv2d_host.argtypes = [_vp, _c_int, _c_int, _vp, _c_int, _c_int, _vp, _c_int, _c_int, _c_int,
+                                   _vp, _c_ll, _vp]
+    lib.sysconv_status_string.restype = ctypes.c_char_p
+    lib.sysconv_status_string.argtypes = [_c_int]
+    lib.sysconv_design_name.restype = ctypes.c_char_p
+    lib.sysconv_design_name.argtypes = [_c_int]
+    lib.sysconv_version.restype = _c_int
+    lib.sysconv_launch_count.restype = _c_ll
+    _lib = lib
+    return lib
+
+
+def status_string(status):
+    if _lib is None:
+        return "library not loaded"
+    return _lib.sysconv_status_string(int(status)).decode()
+
+
+def design_name(design):
+    return load_library().sysconv_design_name(int(design)).decode()
+
+
+def version():
+    return int(load_library().sysconv_version())
+
+
+def launch_count():
+    """Kernels launched by the library in this process so far."""
+    return int(load_library().sysconv_launch_count())
+
+
+def _design(design):
+    if isinstance(design, str):
+        return _DESIGN_BY_NAME[design.upper()]
+    return int(design)
+
+
+def _host_taps(w, dtype, ndim):
+    w = np.ascontiguousarray(w.detach().cpu().numpy() if hasattr(w, "detach") else w,
+                             dtype=np.float32 if dtype == F32 else np.int8)
+    if w.ndim != ndim:
+        raise ValueError("filter must be %d-D" % ndim)
+    return w
+
+
+def _stream_ptr(stream):
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    return int(getattr(stream, "cuda_stream", stream))
+
+
+# ------------------------------------------------------------------ raw C-ABI calls
+
+
+def sysconv1d(x_ptr, n, x_batch_stride, w_host, q, y_ptr, y_batch_stride, batch, dtype, design, stream_ptr):
+    """Raw call: pointers are integers (device x/y, numpy array for the taps). Returns the status."""
+    lib = load_library()
+    return int(lib.sysconv1d(_vp(x_ptr), n, x_batch_stride, w_host.ctypes.data_as(_vp), q, _vp(y_ptr),
+                             y_batch_stride, batch, dtype, design, _vp(stream_ptr)))
+
+
+def sysconv2d(x_ptr, width, height, x_pitch, x_batch_stride, w_host, q, p, y_ptr, y_pitch, y_batch_stride,
+              batch, dtype, design, stream_ptr):
+    lib = load_library()
+    return int(lib.sysconv2d(_vp(x_ptr), width, height, x_pitch, x_batch_stride, w_host.ctypes.data_as(_vp),
+                             q, p, _vp(y_ptr), y_pitch, y_batch_stride, batch, dtype, design,
+                             _vp(stream_ptr)))
+
+
+def host_workspace_bytes(shape, filt, dtype=F32):
+    """Device workspace the *_host entry points need. shape = (n,) | (batch, n) | (h, w) handled by caller."""
+    lib = load_library()
+    if len(filt) == 1:
+        batch, n = (1, shape[0]) if len(shape) == 1 else shape
+        return int(lib.sysconv1d_host_workspace_bytes(n, filt[0], batch, dtype))
+    batch, h, w = (1,) + tuple(shape) if len(shape) == 2 else shape
+    return int(lib.sysconv2d_host_workspace_bytes(w, h, filt[1], filt[0], batch, dtype))
+
+
+def sysconv1d_host(x_host, w_host, y_host, design, workspace, stream=None, dtype=F32):
+    """x_host: (batch, n) or (n,) host array/tensor (pinned for overlap); y_host likewise; workspace: cuda uint8 tensor."""
+    lib = load_library()
+    xs = tuple(x_host.shape)
+    batch, n = (1, xs[0]) if len(xs) == 1 else xs
+    w = _host_taps(w_host, dtype, 1)
+    st = lib.sysconv1d_host(_vp(_data_ptr(x_host)), n, w.ctypes.data_as(_vp), w.shape[0], _vp(_data_ptr(y_host)),
+                            batch, dtype, _design(design), _vp(workspace.data_ptr()), workspace.numel(),
+                            _vp(_stream_ptr(stream)))
+    if st != 0:
+        raise SysconvError(st, "sysconv1d_host")
+
+
+def sysconv2d_host(x_host, w_host, y_host, design, workspace, stream=None, dtype=F32):
+    lib = load_library()
+    xs = tuple(x_host.shape)
+    batch, h, wd = (1,) + xs if len(xs) == 2 else xs
+    w = _host_taps(w_host, dtype, 2)
+    st = lib.sysconv2d_host(_vp(_data_ptr(x_host)), wd, h, w.ctypes.data_as(_vp), w.shape[1], w.shape[0],
+                            _vp(_data_ptr(y_host)), batch, dtype, _design(design), _vp(workspace.data_ptr()),
+                            workspace.numel(), _vp(_stream_ptr(stream)))
+    if st != 0:
+        raise SysconvError(st, "sysconv2d_host")
+
+
+def _data_ptr(a):
+    if hasattr(a, "data_ptr"):
+        return a.data_ptr()
+    return a.ctypes.data
+
+
+# ------------------------------------------------------------------ torch-tensor front end
+
+
+def _dtype_of(x):
+    import torch
+    if x.dtype == torch.float32:
+        return F32, torch.float32
+    if x.dtype == torch.uint8:
+        return U8S8_S32, torch.int32
+    raise TypeError("x must be float32 or uint8, got %s" % x.dtype)
+
+
+def conv1d(x, w, design=OS, out=None, stream=None):
+    """y[b, c] = sum_k w[k] x[b, c+k] on CUDA tensors. x: (n,) or (batch, n), contiguous rows."""
+    import torch
+    if not x.is_cuda:
+        raise SysconvError(-1, "conv1d (x is not a CUDA tensor; there is no CPU path)")
+    dtype, out_dtype = _dtype_of(x)
+    squeeze = x.dim() == 1
+    x2 = x.unsqueeze(0) if squeeze else x
+    if x2.dim() != 2 or x2.stride(1) != 1:
+        raise ValueError("x must be (n,) or (batch, n) with contiguous rows")
+    taps = _host_taps(w, dtype, 1)
+    batch, n = x2.shape
+    q = taps.shape[0]
+    if out is None:
+        out = torch.empty((batch, n - q + 1) if n >= q else (batch, 0), dtype=out_dtype, device=x.device)
+        y2 = out
+    else:
+        y2 = out.unsqueeze(0) if out.dim() == 1 else out
+    st = sysconv1d(x2.data_ptr(), n, x2.stride(0) if batch > 1 else n, taps, q, y2.data_ptr(),
+                   y2.stride(0) if batch > 1 else max(n - q + 1, 0), batch, dtype, _design(design),
+                   _stream_ptr(stream))
+    if st != 0:
+        raise SysconvError(st, "sysconv1d")
+    return out.squeeze(0) if (squeeze and out.dim() == 2) else out
+
+
+def conv2d(x, w, design=OS, out=None, stream=None):
+    """y[b, r, c] = sum_p sum_q w[p, q] x[b, r+p, c+q] on CUDA tensors. x: (h, w) or (batch, h, w)."""
+    import torch
+    if not x.is_cuda:
+        raise SysconvError(-1, "conv2d (x is not a CUDA tensor; there is no CPU path)")
+    dtype, out_dtype = _dtype_of(x)
+    squeeze = x.dim() == 2
+    x3 = x.unsqueeze(0) if squeeze else x
+    if x3.dim() != 3 or x3.stride(2) != 1:
+        raise ValueError("x must be (h, w) or (batch, h, w) with contiguous rows")
+    taps = _host_taps(w, dtype, 2)
+    batch, h, wd = x3.shape
+    p, q = taps.shape
+    if out is None:
+        out = torch.empty((batch, max(h - p + 1, 0), max(wd - q + 1, 0)), dtype=out_dtype, device=x.device)
+        y3 = out
+    else:
+        y3 = out.unsqueeze(0) if out.dim() == 2 else out
+    st = sysconv2d(x3.data_ptr(), wd, h, x3.stride(1), x3.stride(0) if batch > 1 else 0, taps, q, p,
+                   y3.data_ptr(), y3.stride(1), y3.stride(0) if batch > 1 else 0, batch, dtype,
+                   _design(design), _stream_ptr(stream))
+    if st != 0:
+        raise SysconvError(st, "sysconv2d")
+    return out.squeeze(0) if (squeeze and out.dim() == 3) else out

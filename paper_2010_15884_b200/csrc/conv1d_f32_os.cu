@@ -1,0 +1,11 @@
+// 1-D fp32 kernels of the output-stationary (FBS) design, all filter lengths 1..32.
+#include "conv1d_f32.cuh"
+
+namespace sysconv {
+
+cudaError_t launch_conv1d_f32_os(const Conv1DArgs &a, const float *w, int q, cudaStream_t s, int *launches)
+{
+    return launch_conv1d_f32<SYSCONV_OS>(a, w, q, s, launches);
+}
+
+}  // namespace sysconv

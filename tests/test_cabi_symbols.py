@@ -1,0 +1,73 @@
+"""The C-ABI library loads and exports every symbol include/sysconv.h declares (no GPU, no compute)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+HEADER = os.path.join(ROOT, "include", "sysconv.h")
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2010_15884_b200 import build, binding
+    build.build()
+    return binding.load_library()
+
+
+def _declared_functions():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    names = re.findall(r"\b(sysconv\w*)\s*\(", text)
+    return sorted(set(names))
+
+
+def test_header_declares_the_expected_entry_points():
+    names = _declared_functions()
+    for must in ("sysconv1d", "sysconv2d", "sysconv1d_host", "sysconv2d_host", "sysconv_status_string",
+                 "sysconv_design_name", "sysconv_version", "sysconv_launch_count"):
+        assert must in names
+
+
+def test_library_exports_every_declared_symbol(lib):
+    for name in _declared_functions():
+        assert hasattr(lib, name), "libsysconv.so does not export %s" % name
+
+
+def test_strings_and_version_without_a_gpu(lib):
+    from paper_2010_15884_b200 import binding
+    assert binding.version() >= 100
+    assert binding.status_string(0) == "ok"
+    assert binding.status_string(1) == "invalid argument"
+    assert binding.status_string(99) == "?"
+    assert binding.design_name(binding.WS) == "WS/BSM"
+    assert binding.design_name(binding.OS) == "OS/FBS"
+    assert binding.design_name(binding.IS) == "IS/SBM"
+    assert binding.launch_count() >= 0
+
+
+def test_argument_validation_needs_no_gpu(lib):
+    # every one of these is rejected before any CUDA call is made
+    import numpy as np
+    from paper_2010_15884_b200 import binding as b
+    w = np.ones(4, np.float32)
+    fake_x, fake_y = 0x10000, 0x90000000
+    assert b.sysconv1d(0, 100, 100, w, 4, fake_y, 97, 1, b.F32, b.OS, 0) == 1          # null x
+    assert b.sysconv1d(fake_x, 3, 3, w, 4, fake_y, 0, 1, b.F32, b.OS, 0) == 1           # n < q
+    assert b.sysconv1d(fake_x, 100, 100, w, 4, fake_y, 97, 0, b.F32, b.OS, 0) == 1      # batch < 1
+    assert b.sysconv1d(fake_x, 100, 100, w, 4, fake_y, 97, 1, 7, b.OS, 0) == 1          # dtype
+    assert b.sysconv1d(fake_x, 100, 100, w, 4, fake_y, 97, 1, b.F32, 5, 0) == 1         # design
+    assert b.sysconv1d(fake_x, 100, 50, w, 4, fake_y, 97, 2, b.F32, b.OS, 0) == 1       # batch stride < n
+    assert b.sysconv1d(fake_x, 100, 100, w, 4, fake_x + 16, 97, 1, b.F32, b.OS, 0) == 1  # overlap
+    w33 = np.ones(33, np.float32)
+    assert b.sysconv1d(fake_x, 100, 100, w33, 33, fake_y, 68, 1, b.F32, b.OS, 0) == 2   # Q > 32
+    w2 = np.ones((3, 3), np.float32)
+    assert b.sysconv2d(fake_x, 2, 10, 2, 20, w2, 3, 3, fake_y, 8, 64, 1, b.F32, b.OS, 0) == 1    # width < q
+    assert b.sysconv2d(fake_x, 10, 10, 9, 100, w2, 3, 3, fake_y, 8, 64, 1, b.F32, b.OS, 0) == 1  # pitch < width
+    assert b.sysconv2d(fake_x, 10, 10, 10, 100, w2, 3, 3, fake_y, 7, 64, 1, b.F32, b.OS, 0) == 1  # y pitch
+    w16 = np.ones((16, 3), np.float32)
+    assert b.sysconv2d(fake_x, 40, 40, 40, 1600, w16, 3, 16, fake_y, 38, 950, 1, b.F32, b.OS, 0) == 2  # P > 15
+    assert lib.sysconv1d_host_workspace_bytes(100, 4, 2, b.F32) == 1024 + 1024
+    assert lib.sysconv1d_host_workspace_bytes(3, 4, 1, b.F32) == -1
+    assert lib.sysconv2d_host_workspace_bytes(10, 10, 3, 3, 1, b.U8S8_S32) == 256 + 256

@@ -1,0 +1,323 @@
+"""Parity of the CUDA library (through the C ABI) against the CPU oracle, element by element.
+
+fp32: |y_gpu - y_oracle| <= 1e-5 * S with S = sum |w||x| of the same output (the bound stated for
+this build; the oracle accumulates in fp64).  Integer: every int32 equal.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2010_15884_b200 import binding as B
+from paper_2010_15884_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+DESIGNS = [B.WS, B.OS, B.IS]
+TOL = 1e-5
+CANARY = 12345.0
+
+
+def _ids(d):
+    return B.DESIGN_NAMES[d]
+
+
+def assert_close_f32(y_gpu, y_ref, s_ref, what=""):
+    y_gpu = np.asarray(y_gpu, dtype=np.float64)
+    assert y_gpu.shape == y_ref.shape, (y_gpu.shape, y_ref.shape)
+    err = np.abs(y_gpu - y_ref)
+    bound = TOL * s_ref
+    bad = err > bound
+    # outputs whose taps are all zero have S = 0 and must be exactly equal
+    if bad.any():
+        i = np.argmax(err - bound)
+        raise AssertionError("%s: %d outputs beyond 1e-5*S; worst at flat index %d: gpu %r ref %r S %r"
+                             % (what, int(bad.sum()), i, y_gpu.flat[i], y_ref.flat[i], s_ref.flat[i]))
+    assert np.isfinite(y_gpu).all()
+
+
+# ------------------------------------------------------------------------ 1-D fp32
+
+
+def run_1d(x_np, w_np, design, device, batch_stride=None, offset=0):
+    """x_np: (n,) or (batch, n). Returns y as numpy, checks canaries around the output."""
+    x2 = x_np.reshape(1, -1) if x_np.ndim == 1 else x_np
+    batch, n = x2.shape
+    q = w_np.shape[0]
+    n_out = n - q + 1
+    xs = batch_stride or n
+    ys = (batch_stride or n_out)
+    xbuf = torch.zeros(offset + batch * xs + 8, dtype=torch.float32, device=device)
+    ybuf = torch.full((offset + batch * ys + 64,), CANARY, dtype=torch.float32, device=device)
+    for b in range(batch):
+        xbuf[offset + b * xs: offset + b * xs + n] = torch.from_numpy(x2[b]).to(device)
+    st = B.sysconv1d(xbuf.data_ptr() + 4 * offset, n, xs, np.ascontiguousarray(w_np), q,
+                     ybuf.data_ptr() + 4 * offset, ys, batch, B.F32, design,
+                     torch.cuda.current_stream().cuda_stream)
+    assert st == 0, B.status_string(st)
+    torch.cuda.synchronize()
+    yh = ybuf.cpu().numpy()
+    out = np.stack([yh[offset + b * ys: offset + b * ys + n_out] for b in range(batch)])
+    mask = np.ones(yh.shape, bool)
+    for b in range(batch):
+        mask[offset + b * ys: offset + b * ys + n_out] = False
+    assert (yh[mask] == CANARY).all(), "write outside the output range"
+    return out[0] if x_np.ndim == 1 else out
+
+
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+def test_config1_1d_n4096_q8(cuda_device, design):
+    x, ws = inputs.make_config(1)
+    w = ws[8]
+    y_ref, s_ref = oracle.conv1d_f32(x, w)
+    assert y_ref.shape == (4089,)
+    assert_close_f32(run_1d(x, w, design, cuda_device), y_ref, s_ref, "config 1")
+
+
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+@pytest.mark.parametrize("q", list(range(1, 33)))
+def test_1d_every_filter_length(cuda_device, design, q):
+    x, ws = inputs.gen_1d_f32(11000, [q], seed=40 + q)
+    y_ref, s_ref = oracle.conv1d_f32(x, ws[q])
+    assert_close_f32(run_1d(x, ws[q], design, cuda_device), y_ref, s_ref, "q=%d" % q)
+
+
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+@pytest.mark.parametrize("q", [1, 4, 5, 16, 31, 32])
+@pytest.mark.parametrize("extra", [0, 1, 2, 3, 75, 76, 77, 607, 608, 609, 4863, 4864, 4865, 9731])
+def test_1d_ragged_sizes(cuda_device, design, q, extra):
+    n = q + extra           # n_out = extra + 1: single output, tile and warp-tile edges, ragged tails
+    x, ws = inputs.gen_1d_f32(n, [q], seed=1000 + n)
+    y_ref, s_ref = oracle.conv1d_f32(x, ws[q])
+    assert_close_f32(run_1d(x, ws[q], design, cuda_device), y_ref, s_ref, "n=%d q=%d" % (n, q))
+
+
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+@pytest.mark.parametrize("offset", [1, 2, 3])
+def test_1d_unaligned_pointers_and_batch_strides(cuda_device, design, offset):
+    rng = np.random.default_rng(7)
+    x = (rng.random((3, 7001), dtype=np.float32) * 2 - 1).astype(np.float32)
+    w = (rng.random(9, dtype=np.float32) * 2 - 1).astype(np.float32)
+    y = run_1d(x, w, design, cuda_device, batch_stride=7013, offset=offset)
+    for b in range(3):
+        y_ref, s_ref = oracle.conv1d_f32(x[b], w)
+        assert_close_f32(y[b], y_ref, s_ref, "batch %d" % b)
+
+
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+def test_1d_exact_on_small_integers(cuda_device, design):
+    # integer-valued data: every design must reproduce the sums exactly, whatever its order
+    rng = np.random.default_rng(8)
+    x = rng.integers(-50, 51, 30000).astype(np.float32)
+    w = rng.integers(-9, 10, 13).astype(np.float32)
+    y_ref, _ = oracle.conv1d_f32(x, w)
+    np.testing.assert_array_equal(run_1d(x, w, design, cuda_device).astype(np.float64), y_ref)
+
+
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+@pytest.mark.parametrize("q", [4, 16, 32])
+def test_config2_1d_full_size(cuda_device, design, q):
+    """N = 2^26, compared on every output, in the launch configuration bench.py times."""
+    x, ws = inputs.make_config(2)
+    w = ws[q]
+    xd = torch.from_numpy(x).to(cuda_device)
+    yd = B.conv1d(xd, w, design)
+    torch.cuda.synchronize()
+    y_gpu = yd.cpu().numpy()
+    del xd, yd
+    y_ref, s_ref = oracle.conv1d_f32(x, w)
+    assert y_gpu.shape == y_ref.shape == ((1 << 26) - q + 1,)
+    chunk = 1 << 23
+    for lo in range(0, y_ref.size, chunk):
+        hi = min(lo + chunk, y_ref.size)
+        assert_close_f32(y_gpu[lo:hi], y_ref[lo:hi], s_ref[lo:hi], "config 2 q=%d [%d,%d)" % (q, lo, hi))
+
+
+# ------------------------------------------------------------------------ 2-D
+
+
+def run_2d(x_np, w_np, design, device, x_pitch=None, y_pitch=None, x_off=0, y_off=0):
+    """x_np: (batch, h, w) float32 or uint8; returns y (batch, oh, ow); checks canaries."""
+    batch, h, wd = x_np.shape
+    p, q = w_np.shape
+    oh, ow = h - p + 1, wd - q + 1
+    is_f = x_np.dtype == np.float32
+    x_pitch = x_pitch or wd
+    y_pitch = y_pitch or ow
+    xb = torch.zeros(x_off + batch * h * x_pitch + 16, dtype=torch.float32 if is_f else torch.uint8, device=device)
+    canary = CANARY if is_f else 123456789
+    yb = torch.full((y_off + batch * oh * y_pitch + 64,), canary, dtype=torch.float32 if is_f else torch.int32,
+                    device=device)
+    xv = xb[x_off: x_off + batch * h * x_pitch].view(batch, h, x_pitch)
+    xv[:, :, :wd] = torch.from_numpy(x_np).to(device)
+    st = B.sysconv2d(xb.data_ptr() + x_off * xb.element_size(), wd, h, x_pitch, h * x_pitch,
+                     np.ascontiguousarray(w_np), q, p, yb.data_ptr() + y_off * 4, y_pitch, oh * y_pitch, batch,
+                     B.F32 if is_f else B.U8S8_S32, design, torch.cuda.current_stream().cuda_stream)
+    assert st == 0, B.status_string(st)
+    torch.cuda.synchronize()
+    yh = yb.cpu().numpy()
+    body = yh[y_off: y_off + batch * oh * y_pitch].reshape(batch, oh, y_pitch)
+    out = body[:, :, :ow].copy()
+    assert (body[:, :, ow:] == canary).all(), "write into the pitch padding"
+    assert (yh[:y_off] == canary).all() and (yh[y_off + batch * oh * y_pitch:] == canary).all()
+    return out
+
+
+def check_2d(x_np, w_np, design, device, **kw):
+    y = run_2d(x_np, w_np, design, device, **kw)
+    for b in range(x_np.shape[0]):
+        if x_np.dtype == np.float32:
+            y_ref, s_ref = oracle.conv2d_f32(x_np[b], w_np)
+            assert_close_f32(y[b], y_ref, s_ref, "image %d" % b)
+        else:
+            np.testing.assert_array_equal(y[b], oracle.conv2d_u8s8_s32(x_np[b], w_np))
+
+
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+def test_config3_2d_1920x1080_5x5(cuda_device, design):
+    x, ws = inputs.make_config(3)
+    check_2d(x, ws[(5, 5)], design, cuda_device)
+
+
+FILTERS_2D = [(1, 1), (1, 5), (5, 1), (2, 2), (3, 3), (5, 5), (7, 7), (9, 9), (15, 15), (2, 11), (13, 4), (15, 1),
+              (1, 15), (8, 6)]
+
+
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+@pytest.mark.parametrize("pq", FILTERS_2D, ids=lambda f: "%dx%d" % f)
+def test_2d_f32_filter_shapes(cuda_device, design, pq):
+    p, q = pq
+    x, ws = inputs.gen_2d_f32(300, 75, [pq], seed=50 + p * 16 + q, batch=2)
+    check_2d(x, ws[pq], design, cuda_device)
+
+
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+@pytest.mark.parametrize("hw", [(0, 0), (1, 0), (0, 1), (2, 3), (31, 127), (32, 128), (33, 129), (40, 255), (7, 513)])
+@pytest.mark.parametrize("pq", [(3, 3), (5, 7), (15, 15)], ids=lambda f: "%dx%d" % f)
+def test_2d_f32_ragged_image_sizes(cuda_device, design, hw, pq):
+    # output sizes (hw[0]+1) x (hw[1]+1): single output, strip/band edges, ragged tails
+    p, q = pq
+    x, ws = inputs.gen_2d_f32(q + hw[1], p + hw[0], [pq], seed=77 + hw[0] + hw[1])
+    check_2d(x, ws[pq], design, cuda_device)
+
+
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+@pytest.mark.parametrize("pitches", [(203, 199, 1, 1), (204, 198, 0, 2), (201, 200, 3, 0), (208, 196, 4, 4)])
+def test_2d_f32_pitches_and_alignment(cuda_device, design, pitches):
+    xp, yp, xo, yo = pitches
+    x, ws = inputs.gen_2d_f32(200, 41, [(5, 5)], seed=91, batch=2)
+    check_2d(x, ws[(5, 5)], design, cuda_device, x_pitch=xp, y_pitch=yp, x_off=xo, y_off=yo)
+
+
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+@pytest.mark.parametrize("k", [3, 9, 15])
+def test_config5_reduced_and_exact_integers(cuda_device, design, k):
+    x, ws = inputs.make_config(5, scale=dict(width=520, height=300, batch=2, filters=[k]))
+    check_2d(x, ws[(k, k)], design, cuda_device)
+    rng = np.random.default_rng(k)
+    xi = rng.integers(0, 16, (1, 100, 260)).astype(np.float32)
+    wi = rng.integers(-4, 5, (k, k)).astype(np.float32)
+    y = run_2d(xi, wi, design, cuda_device)
+    np.testing.assert_array_equal(y[0].astype(np.float64), oracle.conv2d_f32(xi[0], wi)[0])
+
+
+@pytest.mark.parametrize("k", [3, 9, 15])
+def test_config5_full_size_sampled(cuda_device, k):
+    """16 x 4096 x 4096 in the bench's launch configuration; sampled outputs against the oracle."""
+    x, ws = inputs.make_config(5, scale=dict(filters=[k]))
+    w = ws[(k, k)]
+    xd = torch.from_numpy(x).to(cuda_device)
+    rng = np.random.default_rng(5)
+    oh = ow = 4096 - k + 1
+    rows = np.concatenate([rng.integers(0, oh, 4000), [0, 0, oh - 1, oh - 1]]).astype(np.int64)
+    cols = np.concatenate([rng.integers(0, ow, 4000), [0, ow - 1, 0, ow - 1]]).astype(np.int64)
+    yd = torch.empty((16, oh, ow), dtype=torch.float32, device=cuda_device)
+    for design in DESIGNS:
+        yd.fill_(CANARY)
+        B.conv2d(xd, w, design, out=yd)
+        torch.cuda.synchronize()
+        ri, ci = torch.from_numpy(rows).to(cuda_device), torch.from_numpy(cols).to(cuda_device)
+        for b in range(16):
+            got = yd[b][ri, ci].cpu().numpy()
+            y_ref, s_ref = oracle.conv2d_f32_at(x[b], w, rows, cols)
+            assert_close_f32(got, y_ref, s_ref, "config 5 k=%d design %s image %d" % (k, _ids(design), b))
+        # every output was written (no canary left) and the whole of image 7 matches at k = 3
+        assert not bool((yd == CANARY).any())
+        if k == 3:
+            y_ref, s_ref = oracle.conv2d_f32(x[7], w)
+            assert_close_f32(yd[7].cpu().numpy(), y_ref, s_ref, "config 5 image 7 full")
+
+
+# ------------------------------------------------------------------------ integer
+
+
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+@pytest.mark.parametrize("k", [3, 7])
+def test_config4_2d_u8_full(cuda_device, design, k):
+    x, ws = inputs.make_config(4, scale=dict(filters=[k]))
+    check_2d(x, ws[(k, k)], design, cuda_device)
+
+
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+@pytest.mark.parametrize("pq", [(1, 1), (3, 3), (7, 7), (2, 5), (15, 15), (4, 13)], ids=lambda f: "%dx%d" % f)
+def test_2d_u8_shapes_and_extremes(cuda_device, design, pq):
+    p, q = pq
+    x, ws = inputs.gen_2d_u8s8(301, 67, [pq], seed=60 + p + q, batch=2)
+    check_2d(x, ws[pq], design, cuda_device)
+    check_2d(x, ws[pq], design, cuda_device, x_pitch=307, y_pitch=303, x_off=1, y_off=1)
+    xm = np.full((1, 40, 150), 255, np.uint8)
+    for v in (8, -8):
+        check_2d(xm, np.full(pq, v, np.int8), design, cuda_device)
+
+
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+def test_1d_u8(cuda_device, design):
+    x, ws = inputs.gen_1d_u8s8(5000, [7], seed=3)
+    xd = torch.from_numpy(x).to(cuda_device)
+    y = B.conv1d(xd, ws[7], design)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(y.cpu().numpy(), oracle.conv1d_u8s8_s32(x, ws[7]))
+
+
+# ------------------------------------------------------------------------ host-buffer entry points
+
+
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+def test_host_entry_points(cuda_device, design):
+    x, ws = inputs.gen_1d_f32(100000, [16], seed=21)
+    xh = torch.from_numpy(x).pin_memory()
+    yh = torch.empty(100000 - 15, dtype=torch.float32).pin_memory()
+    wsz = B.host_workspace_bytes((100000,), (16,))
+    work = torch.empty(wsz, dtype=torch.uint8, device=cuda_device)
+    B.sysconv1d_host(xh, ws[16], yh, design, work)
+    torch.cuda.synchronize()
+    y_ref, s_ref = oracle.conv1d_f32(x, ws[16])
+    assert_close_f32(yh.numpy(), y_ref, s_ref, "1-D host")
+    small = torch.empty(wsz - 256, dtype=torch.uint8, device=cuda_device)
+    with pytest.raises(B.SysconvError):
+        B.sysconv1d_host(xh, ws[16], yh, design, small)
+
+    x2, ws2 = inputs.gen_2d_u8s8(333, 222, [(3, 3)], seed=22, batch=2)
+    xh2 = torch.from_numpy(x2).pin_memory()
+    yh2 = torch.empty((2, 220, 331), dtype=torch.int32).pin_memory()
+    work2 = torch.empty(B.host_workspace_bytes((2, 222, 333), (3, 3), B.U8S8_S32), dtype=torch.uint8,
+                        device=cuda_device)
+    B.sysconv2d_host(xh2, ws2[(3, 3)], yh2, design, work2, dtype=B.U8S8_S32)
+    torch.cuda.synchronize()
+    for b in range(2):
+        np.testing.assert_array_equal(yh2[b].numpy(), oracle.conv2d_u8s8_s32(x2[b], ws2[(3, 3)]))
+
+
+def test_unsupported_and_invalid_on_device(cuda_device):
+    x = torch.zeros(1000, device=cuda_device)
+    with pytest.raises(B.SysconvError) as e:
+        B.conv1d(x, np.ones(33, np.float32))
+    assert e.value.status == 2
+    with pytest.raises(B.SysconvError) as e:
+        B.conv1d(x[:5], np.ones(8, np.float32), out=torch.zeros(8, device=cuda_device))
+    assert e.value.status == 1
+    with pytest.raises(B.SysconvError):
+        B.conv1d(torch.zeros(10), np.ones(3, np.float32))     # CPU tensor: no fallback
+    before = B.launch_count()
+    B.conv1d(x, np.ones(8, np.float32))
+    assert B.launch_count() == before + 1
