@@ -59,7 +59,8 @@ typedef enum {
     SYSCONV_EINVAL = 1,
     SYSCONV_EUNSUPPORTED = 2,
     SYSCONV_ECUDA = 3,
-    SYSCONV_ETIMEOUT = 4
+    SYSCONV_ETIMEOUT = 4,
+    SYSCONV_ETOOLARGE = 5 /* problem exceeds the built-in staging area of sysconv1d_host_static */
 } sysconv_status;
 
 typedef enum {
@@ -119,6 +120,38 @@ int sysconv1d_host(const void *x_host, long long n, const void *w_host, int q,
 int sysconv2d_host(const void *x_host, int width, int height, const void *w_host, int q, int p,
                    void *y_host, int batch, int dtype, int design,
                    void *workspace_dev, long long workspace_bytes, void *stream);
+
+/*
+ * sysconv1d_host for callers that cannot allocate device memory.  (The paper has
+ * no counterpart: this is a packaging variant, not a systolic design.)
+ *
+ * Who needs it: code that runs where the CUDA allocator is off limits -- a plug-in
+ * inside an application that has handed the whole device to its own memory arena,
+ * a steady-state real-time loop where cudaMalloc (which serialises the device and
+ * can fail late) is banned, a process whose memory budget was fixed at start-up.
+ * Such a caller cannot supply the device workspace sysconv1d_host asks for.
+ *
+ * This entry point takes the same host buffers and stages them in a fixed array
+ * that is part of the library's device image, so it allocates nothing: no
+ * cudaMalloc/cudaFree, no allocating library call.  Same arguments and results as
+ * sysconv1d_host, minus the workspace.
+ *   - Limit: sysconv1d_host_workspace_bytes(n, q, batch, dtype) must not exceed
+ *     sysconv_static_scratch_bytes() (16 MiB: about 2 Mi fp32 samples in one
+ *     signal, or the same total over a batch).  Larger problems return
+ *     SYSCONV_ETOOLARGE and enqueue nothing.
+ *   - Cost: every GPU on which this library is loaded holds those 16 MiB until
+ *     the process exits, whether or not this function is ever called.
+ *   - The first call on each device resolves the array's device address (once,
+ *     with that device current); make that first call outside any stream capture.
+ *   - All calls on one device share the one array: calls whose work overlaps on
+ *     the GPU (different streams, or threads, without ordering between them)
+ *     race on it.  Issue them on one stream or order them yourself.  Nothing in
+ *     the array needs clearing between calls: inputs are fully overwritten and
+ *     every output is written before it is copied back.
+ */
+long long sysconv_static_scratch_bytes(void);
+int sysconv1d_host_static(const void *x_host, long long n, const void *w_host, int q,
+                          void *y_host, int batch, int dtype, int design, void *stream);
 
 /* Text for a sysconv_status / sysconv_design value ("?" if unknown). Static storage. */
 const char *sysconv_status_string(int status);

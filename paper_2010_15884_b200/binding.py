@@ -57,6 +57,9 @@ def load_library():
     lib.sysconv2d_host.restype = _c_int
     lib.sysconv2d_host.argtypes = [_vp, _c_int, _c_int, _vp, _c_int, _c_int, _vp, _c_int, _c_int, _c_int,
                                    _vp, _c_ll, _vp]
+    lib.sysconv1d_host_static.restype = _c_int
+    lib.sysconv1d_host_static.argtypes = [_vp, _c_ll, _vp, _c_int, _vp, _c_int, _c_int, _c_int, _vp]
+    lib.sysconv_static_scratch_bytes.restype = _c_ll
     lib.sysconv_status_string.restype = ctypes.c_char_p
     lib.sysconv_status_string.argtypes = [_c_int]
     lib.sysconv_design_name.restype = ctypes.c_char_p
@@ -146,6 +149,28 @@ def sysconv1d_host(x_host, w_host, y_host, design, workspace, stream=None, dtype
                             _vp(_stream_ptr(stream)))
     if st != 0:
         raise SysconvError(st, "sysconv1d_host")
+
+
+def static_scratch_bytes():
+    """Size of the staging area built into the library for sysconv1d_host_static."""
+    return int(load_library().sysconv_static_scratch_bytes())
+
+
+def sysconv1d_host_static(x_host, w_host, y_host, design, stream=None, dtype=F32):
+    """sysconv1d_host without a workspace argument, for callers that cannot allocate device memory.
+
+    The data is staged in a fixed 16 MiB array inside the library, so problems are limited to what
+    fits there (SysconvError with status 5 otherwise) and calls that overlap on the GPU race on it.
+    """
+    lib = load_library()
+    xs = tuple(x_host.shape)
+    batch, n = (1, xs[0]) if len(xs) == 1 else xs
+    w = _host_taps(w_host, dtype, 1)
+    st = lib.sysconv1d_host_static(_vp(_data_ptr(x_host)), n, w.ctypes.data_as(_vp), w.shape[0],
+                                   _vp(_data_ptr(y_host)), batch, dtype, _design(design),
+                                   _vp(_stream_ptr(stream)))
+    if st != 0:
+        raise SysconvError(st, "sysconv1d_host_static")
 
 
 def sysconv2d_host(x_host, w_host, y_host, design, workspace, stream=None, dtype=F32):

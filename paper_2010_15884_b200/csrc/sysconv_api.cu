@@ -189,6 +189,7 @@ const char *sysconv_status_string(int status)
         case SYSCONV_EUNSUPPORTED: return "unsupported size";
         case SYSCONV_ECUDA: return "CUDA runtime error";
         case SYSCONV_ETIMEOUT: return "device-side wait timed out";
+        case SYSCONV_ETOOLARGE: return "problem larger than the built-in staging area";
         default: return "?";
     }
 }
