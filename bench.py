@@ -305,7 +305,12 @@ def run_ours(args):
     hbm_gbs, peak_kind, sm_max = measured_peaks()
 
     cfg_id = int(args.workload.replace("cfg", ""))
-    cases, keep = build_cases(cfg_id, device)          # every rank holds its own copy: weak scaling
+    scale = None
+    if args.profile_n and cfg_id in (1, 2):
+        scale = {"n": args.profile_n}                  # reduced case for ncu captures only
+    if args.profile_batch and cfg_id == 5:
+        scale = {"batch": args.profile_batch}
+    cases, keep = build_cases(cfg_id, device, scale=scale)   # every rank holds its own copy: weak scaling
     outputs_per_step = sum(c.n_out for c in cases)
 
     # ---- device-resident timing: W warm-up steps, then exactly K timed steps
@@ -362,7 +367,7 @@ def run_ours(args):
     }
 
     # ---- end to end through the host-buffer entry points (rank-local pinned buffers)
-    e2e = run_e2e(cfg_id, device, args, world)
+    e2e = None if (args.no_e2e or scale) else run_e2e(cfg_id, device, args, world)
 
     line = {
         "metric": "output elements/s", "value": round(value, 3), "unit": "Gpix/s", "n_gpus": world,
@@ -378,10 +383,13 @@ def run_ours(args):
         "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
     }
     if rank == 0:
-        outs, secs, cores, what = oracle_sample(cfg_id)
-        line["cpu_baseline"] = {
-            "value": round(outs / secs / 1e9, 4), "unit": "Gpix/s", "cores": cores, "kind": "oracle",
-            "sample": "%s of configuration %d (%.1f s)" % (what, cfg_id, secs)}
+        if scale:
+            line["config"]["reduced_for_profiling"] = scale
+        if not args.no_cpu:
+            outs, secs, cores, what = oracle_sample(cfg_id)
+            line["cpu_baseline"] = {
+                "value": round(outs / secs / 1e9, 4), "unit": "Gpix/s", "cores": cores, "kind": "oracle",
+                "sample": "%s of configuration %d (%.1f s)" % (what, cfg_id, secs)}
         line["per_kernel"] = detail_rows(cases, hbm_gbs, peak_kind, sm_max)
         if not args.no_detail and world == 1:
             del cases, keep
@@ -487,6 +495,12 @@ def main():
     ap.add_argument("--no-detail", action="store_true", help="skip the per-kernel table of the other configurations")
     ap.add_argument("--detail-reps", type=int, default=10)
     ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--profile-n", type=int, default=0,
+                    help="ncu captures only: shrink the 1-D signal to this many samples (keep it > L2)")
+    ap.add_argument("--profile-batch", type=int, default=0,
+                    help="ncu captures only: shrink configuration 5 to this many images")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3

@@ -157,6 +157,16 @@ int sysconv1d_host_static(const void *x_host, long long n, const void *w_host, i
 const char *sysconv_status_string(int status);
 const char *sysconv_design_name(int design);
 
+/*
+ * Device-side health check.  The pipelined kernels wait for their asynchronous
+ * copies with a bounded number of polls; a kernel whose limit runs out stops
+ * taking work, raises a flag in device memory and returns normally (its outputs
+ * are then incomplete).  This call synchronises the current device with a
+ * blocking copy, returns SYSCONV_ETIMEOUT if the flag was raised since the last
+ * call (and clears it), SYSCONV_OK otherwise.
+ */
+int sysconv_device_status(void);
+
 /* Library version, major*10000 + minor*100 + patch. */
 int sysconv_version(void);
 

@@ -65,6 +65,7 @@ def load_library():
     lib.sysconv_design_name.restype = ctypes.c_char_p
     lib.sysconv_design_name.argtypes = [_c_int]
     lib.sysconv_version.restype = _c_int
+    lib.sysconv_device_status.restype = _c_int
     lib.sysconv_launch_count.restype = _c_ll
     _lib = lib
     return lib
@@ -82,6 +83,11 @@ def design_name(design):
 
 def version():
     return int(load_library().sysconv_version())
+
+
+def device_status():
+    """0 if no kernel gave up a bounded wait on the current device since the last call, else 4 (time-out)."""
+    return int(load_library().sysconv_device_status())
 
 
 def launch_count():

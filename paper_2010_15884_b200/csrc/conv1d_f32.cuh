@@ -1,84 +1,70 @@
 // 1-D fp32 convolution (Eq. 2) as folded linear systolic arrays on a warp.
 //
-// One CTA handles one tile of kTileOut1 outputs: it stages the kTileIn1 inputs
-// the tile needs in shared memory, each of its 8 warps runs one systolic array
-// pass over its 640-input slice (608 outputs), the outputs are collected in
-// shared memory and leave with coalesced 128-bit stores.
+// One CTA handles K consecutive tiles of outputs.  Thread 0 fetches the inputs each tile needs with one
+// bulk asynchronous copy per tile (global -> shared, completion on the tile's mbarrier), all K copies
+// issued up front; every warp waits for a tile, runs its systolic array pass on its slice, collects its
+// outputs in shared memory and its lane 0 sends them to global memory with one bulk copy, then moves
+// to the next tile, whose copy has meanwhile landed.  No thread spends instructions on staging.
 //
-// Lane l of a warp holds the R1 = 20 consecutive PEs l*20 .. l*20+19.  A time
-// step is R1 fused multiply-adds per lane, one shuffle (the value that crosses
-// the lane boundary) and a renaming of the lane's own registers (the loops over
-// time are fully unrolled, so "PE j takes PE j-1's value" costs nothing).
-// Every PE runs at every step (no CheckTime); PEs whose sums are incomplete are
-// not drained.
+// CTAs are small and each takes a fixed, contiguous piece of the signal, on purpose: on B200 the
+// in-order CTA dispatcher keeps reads and writes evenly mixed and sustains ~6.2 TB/s, where persistent
+// grid-stride loops over the same tiles (bulk copies or plain loads alike) stalled near 5.5 TB/s.
+//
+// Tiles that touch the end of the signal, and calls whose x or y is not 16-byte aligned, are staged
+// with ordinary loads/stores by the threads of the CTA instead (same kernel, same passes).
+//
+// Lane l of a warp holds R1 = 20 consecutive PEs.  A time step is R1 fused multiply-adds per lane, one
+// shuffle (the value that crosses the lane boundary) and a renaming of the lane's own registers (the
+// loops over time are fully unrolled, so "PE j takes PE j-1's value" costs nothing).  Every PE runs at
+// every step (no CheckTime); PEs whose sums are incomplete are not drained.
+//
+// The waits on the mbarriers are bounded; if a limit runs out the CTA raises *status_word, gives its
+// other copies a bounded chance to land and returns without writing the rest of its tiles.
 #pragma once
 
 #include "sysconv_common.cuh"
+#include "tma_utils.cuh"
 
 namespace sysconv {
 
-// ---- tile staging -----------------------------------------------------------
+// Tile geometry of a design.  OS and IS: each warp turns 640 inputs into 608 outputs.  WS: each warp
+// holds 16 two-lane arrays that stream 76 outputs each (1216 outputs per warp).  A tile is WARPS
+// warp slices plus a 32-element halo (the halo budget is 32 whatever Q).
+template <int DESIGN, int WARPS>
+struct Geo1D {
+    static constexpr int kWarps = WARPS;
+    static constexpr int kWarpOut = DESIGN == SYSCONV_WS ? kWsArrays1 * kWsSeg1 : kWarpOut1;
+    static constexpr int kThreads = kWarps * kLanes;
+    static constexpr int kTileOut = kWarps * kWarpOut;     // outputs per CTA tile
+    static constexpr int kTileIn = kTileOut + kHalo1;      // inputs per CTA tile
+};
+// shape used by the library (measured best on B200): OS/IS two warps and two tiles per CTA,
+// WS one warp and one (twice as large) tile per CTA
+template <int DESIGN>
+struct DefaultShape1D {
+    static constexpr int kWarps = DESIGN == SYSCONV_WS ? 1 : 2;
+    static constexpr int kTiles = DESIGN == SYSCONV_WS ? 1 : 2;
+};
 
-// Copy x[t0 .. t0 + kTileIn1) to shared memory, zeros beyond the signal's end.
+// ---- ordinary-load staging (ragged or unaligned tiles) ------------------------
+
+// Copy x[t0 .. t0 + tile_in) to shared memory, zeros beyond the signal's end.
 __device__ __forceinline__ void stage_in_1d(const float *__restrict__ xg, long long n, long long t0,
-                                            float *s_in)
+                                            float *s_in, int tile_in, int threads)
 {
-    const bool vec_ok = (reinterpret_cast<uintptr_t>(xg) & 15) == 0;   // t0 is a multiple of 4
-    if (vec_ok) {
-        constexpr int kVec = kTileIn1 / 4;
-        constexpr int kIter = (kVec + kThreads1 - 1) / kThreads1;
-        float4 v[kIter];
-#pragma unroll
-        for (int it = 0; it < kIter; ++it) {
-            const int i = threadIdx.x + it * kThreads1;
-            const long long g = t0 + 4LL * i;
-            v[it] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (i < kVec) {
-                if (g + 3 < n) {
-                    v[it] = __ldg(reinterpret_cast<const float4 *>(xg + g));
-                } else {
-                    if (g < n) v[it].x = xg[g];
-                    if (g + 1 < n) v[it].y = xg[g + 1];
-                    if (g + 2 < n) v[it].z = xg[g + 2];
-                }
-            }
-        }
-#pragma unroll
-        for (int it = 0; it < kIter; ++it) {
-            const int i = threadIdx.x + it * kThreads1;
-            if (i < kVec) reinterpret_cast<float4 *>(s_in)[i] = v[it];
-        }
-    } else {
-        for (int i = threadIdx.x; i < kTileIn1; i += kThreads1) {
-            const long long g = t0 + i;
-            s_in[i] = g < n ? xg[g] : 0.f;
-        }
+    for (int i = threadIdx.x; i < tile_in; i += threads) {
+        const long long g = t0 + i;
+        s_in[i] = g < n ? xg[g] : 0.f;
     }
 }
 
-// Copy the tile's outputs from shared memory to y[t0 .. min(t0 + kTileOut1, n_out)).
+// Copy the tile's outputs from shared memory to y[t0 .. min(t0 + tile_out, n_out)).
 __device__ __forceinline__ void stage_out_1d(float *__restrict__ yg, long long n_out, long long t0,
-                                             const float *s_out)
+                                             const float *s_out, int tile_out, int threads)
 {
-    const bool vec_ok = (reinterpret_cast<uintptr_t>(yg) & 15) == 0;
-    if (vec_ok) {
-        constexpr int kVec = kTileOut1 / 4;
-        for (int i = threadIdx.x; i < kVec; i += kThreads1) {
-            const long long g = t0 + 4LL * i;
-            const float4 v = reinterpret_cast<const float4 *>(s_out)[i];
-            if (g + 3 < n_out) {
-                *reinterpret_cast<float4 *>(yg + g) = v;
-            } else {
-                if (g < n_out) yg[g] = v.x;
-                if (g + 1 < n_out) yg[g + 1] = v.y;
-                if (g + 2 < n_out) yg[g + 2] = v.z;
-            }
-        }
-    } else {
-        for (int i = threadIdx.x; i < kTileOut1; i += kThreads1) {
-            const long long g = t0 + i;
-            if (g < n_out) yg[g] = s_out[i];
-        }
+    for (int i = threadIdx.x; i < tile_out; i += threads) {
+        const long long g = t0 + i;
+        if (g < n_out) yg[g] = s_out[i];
     }
 }
 
@@ -157,16 +143,18 @@ __device__ __forceinline__ void is_pass_1d(const float *sx, float *so, const Tap
 // ---- weight-stationary (BSM, Table 2): PE s keeps w(s); at step t the input
 // x(t) is broadcast to the array, Z_s <- Z_{s-1} + x(t) * w(s), PE 0 starts a new
 // sum and the last PE emits y(t-(Q-1)).  An array has only Q PEs, so a warp holds
-// eight arrays of four lanes (RW = ceil(Q/4) PEs per lane, unused PEs keep a zero
-// tap); array a streams the 76-output segment a of the warp tile.
+// sixteen arrays of two lanes (RW PEs per lane, unused PEs keep a zero tap; the
+// array length QP = 2*RW is kept a multiple of four so that outputs leave as
+// aligned 128-bit words); array a streams the 76-output segment a of the warp's
+// 1216-output slice.  The broadcast is a same-address shared-memory read.
 template <int Q>
 __device__ __forceinline__ void ws_pass_1d(const float *sx, float *so, const Taps1D &taps, int lane)
 {
-    constexpr int RW = (Q + kWsLanes - 1) / kWsLanes;
-    constexpr int QP = RW * kWsLanes;
+    constexpr int RW = 2 * ((Q + 3) / 4);
+    constexpr int QP = RW * kWsLanes1;
     constexpr int kGroups = (kWsSeg1 + QP) / 4;       // time steps in groups of four
-    const int m = lane & (kWsLanes - 1);
-    const int arr = lane / kWsLanes;
+    const int m = lane & (kWsLanes1 - 1);
+    const int arr = lane / kWsLanes1;
     float Wr[RW], Z[RW];
 #pragma unroll
     for (int i = 0; i < RW; ++i) {
@@ -178,7 +166,7 @@ __device__ __forceinline__ void ws_pass_1d(const float *sx, float *so, const Tap
     float *yo = so + arr * kWsSeg1;
 
     auto step = [&](float xb) -> float {
-        float up = __shfl_up_sync(kFullMask, Z[RW - 1], 1, kWsLanes);
+        float up = __shfl_up_sync(kFullMask, Z[RW - 1], 1, kWsLanes1);
         if (m == 0) up = 0.f;                          // PE 0: Z starts at zero
 #pragma unroll
         for (int i = RW - 1; i > 0; --i) Z[i] = fmaf(xb, Wr[i], Z[i - 1]);
@@ -187,64 +175,122 @@ __device__ __forceinline__ void ws_pass_1d(const float *sx, float *so, const Tap
     };
 
     float o0 = 0.f;
-#pragma unroll 2
+#pragma unroll
     for (int k = 0; k < kGroups; ++k) {
         const float4 xv = xs4[k];                      // x(4k .. 4k+3) of this array's stream
         const float o1 = step(xv.x);
         const float o2 = step(xv.y);
         const float o3 = step(xv.z);
         const int off = 4 * k - QP;                    // outputs 4k-QP .. 4k-QP+3 are now complete
-        if (m == kWsLanes - 1 && off >= 0 && off < kWsSeg1)
+        if (m == kWsLanes1 - 1 && off >= 0 && off < kWsSeg1)
             *reinterpret_cast<float4 *>(yo + off) = make_float4(o0, o1, o2, o3);
         o0 = step(xv.w);
     }
 }
 
-template <int DESIGN, int Q>
-__global__ void __launch_bounds__(kThreads1)
-conv1d_f32_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps)
+template <int DESIGN, int Q, int WARPS, int K>
+__global__ void __launch_bounds__(Geo1D<DESIGN, WARPS>::kThreads)
+conv1d_f32_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, unsigned *status_word)
 {
-    __shared__ __align__(16) float s_in[kTileIn1];
-    __shared__ __align__(16) float s_out[kTileOut1];
+    using G = Geo1D<DESIGN, WARPS>;
+    __shared__ __align__(128) float s_in[K][G::kTileIn];
+    __shared__ __align__(128) float s_out[K][G::kTileOut];
+    __shared__ __align__(8) uint64_t full[K];
     const int lane = threadIdx.x & (kLanes - 1);
     const int warp = threadIdx.x / kLanes;
-    const long long t0 = static_cast<long long>(blockIdx.x) * kTileOut1;
+    const long long base = static_cast<long long>(blockIdx.x) * (K * G::kTileOut);
+    // bulk copies need 16-byte aligned global addresses (tile starts are multiples of 4 elements)
+    const bool x_ok = ((reinterpret_cast<uintptr_t>(a.x) & 15) == 0) && (a.batch == 1 || (a.x_bstride & 3) == 0);
+    const bool y_ok = ((reinterpret_cast<uintptr_t>(a.y) & 15) == 0) && (a.batch == 1 || (a.y_bstride & 3) == 0);
 
+    if (threadIdx.x == 0) {
+        for (int k = 0; k < K; ++k) mbar_init(&full[k], 1);
+        mbar_init_fence();
+    }
+    unsigned phase = 0;
     for (int b = blockIdx.y; b < a.batch; b += gridDim.y) {
         const float *xg = static_cast<const float *>(a.x) + b * a.x_bstride;
         float *yg = static_cast<float *>(a.y) + b * a.y_bstride;
-        stage_in_1d(xg, a.n, t0, s_in);
+        // the barriers are initialised, and all warps are done with the previous signal's tiles
         __syncthreads();
-        const float *sx = s_in + warp * kWarpOut1;
-        float *so = s_out + warp * kWarpOut1;
-        if (DESIGN == SYSCONV_OS) os_pass_1d<Q>(sx, so, taps, lane);
-        else if (DESIGN == SYSCONV_IS) is_pass_1d<Q>(sx, so, taps, lane);
-        else ws_pass_1d<Q>(sx, so, taps, lane);
-        __syncthreads();
-        stage_out_1d(yg, a.n_out, t0, s_out);
-        // the next batch iteration's stage_in writes s_in only; s_out is rewritten
-        // after its __syncthreads, when every thread has finished stage_out
+        if (threadIdx.x == 0) {
+#pragma unroll
+            for (int k = 0; k < K; ++k) {
+                const long long t0 = base + k * G::kTileOut;
+                if (x_ok && t0 + G::kTileIn <= a.n) {
+                    mbar_arrive_expect_tx(&full[k], G::kTileIn * 4);
+                    bulk_load(s_in[k], xg + t0, G::kTileIn * 4, &full[k]);
+                }
+            }
+        }
+#pragma unroll 1
+        for (int k = 0; k < K; ++k) {
+            const long long t0 = base + k * G::kTileOut;
+            if (t0 >= a.n_out) break;
+            const bool in_by_copy = x_ok && t0 + G::kTileIn <= a.n;
+            const bool out_by_copy = y_ok && t0 + G::kTileOut <= a.n_out;
+            if (in_by_copy) {
+                const bool ok = mbar_wait_bounded(&full[k], phase);
+                const bool give_up = WARPS == 1 ? __any_sync(kFullMask, !ok) != 0 : __syncthreads_or(!ok) != 0;
+                if (give_up) {
+                    if (threadIdx.x == 0) {
+                        atomicExch(status_word, 1u);
+                        for (int j = k + 1; j < K; ++j)      // copies still in flight target this CTA's memory
+                            if (x_ok && base + j * G::kTileOut + G::kTileIn <= a.n)
+                                mbar_wait_bounded(&full[j], phase, 1u << 16);
+                        bulk_wait_read<0>();
+                    }
+                    return;
+                }
+            } else {
+                stage_in_1d(xg, a.n, t0, s_in[k], G::kTileIn, G::kThreads);
+                __syncthreads();
+            }
+
+            const float *sx = s_in[k] + warp * G::kWarpOut;
+            float *so = s_out[k] + warp * G::kWarpOut;
+            if (DESIGN == SYSCONV_OS) os_pass_1d<Q>(sx, so, taps, lane);
+            else if (DESIGN == SYSCONV_IS) is_pass_1d<Q>(sx, so, taps, lane);
+            else ws_pass_1d<Q>(sx, so, taps, lane);
+
+            if (out_by_copy) {
+                fence_proxy_async();                     // my shared-memory writes, before the bulk store reads them
+                __syncwarp();
+                if (lane == 0) {
+                    bulk_store(yg + t0 + warp * G::kWarpOut, so, G::kWarpOut * 4);
+                    bulk_commit();
+                }
+            } else {
+                __syncthreads();
+                stage_out_1d(yg, a.n_out, t0, s_out[k], G::kTileOut, G::kThreads);
+            }
+        }
+        phase ^= 1u;
+        if (lane == 0) bulk_wait_read<0>();              // shared memory may be reused (or released) after this
     }
 }
 
-template <int DESIGN, int Q>
-cudaError_t launch_conv1d_f32_q(const Conv1DArgs &a, const Taps1D &taps, cudaStream_t s)
+template <int DESIGN, int Q, int WARPS = DefaultShape1D<DESIGN>::kWarps, int K = DefaultShape1D<DESIGN>::kTiles>
+cudaError_t launch_conv1d_f32_q(const Conv1DArgs &a, const Taps1D &taps, unsigned *status_word, cudaStream_t s)
 {
-    const long long tiles = (a.n_out + kTileOut1 - 1) / kTileOut1;
-    if (tiles > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
-    dim3 grid(static_cast<unsigned>(tiles), static_cast<unsigned>(a.batch < 65535 ? a.batch : 65535));
-    conv1d_f32_kernel<DESIGN, Q><<<grid, kThreads1, 0, s>>>(a, taps);
+    using G = Geo1D<DESIGN, WARPS>;
+    const long long per_cta = static_cast<long long>(K) * G::kTileOut;
+    const long long ctas = (a.n_out + per_cta - 1) / per_cta;
+    if (ctas > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    dim3 grid(static_cast<unsigned>(ctas), static_cast<unsigned>(a.batch < 65535 ? a.batch : 65535));
+    conv1d_f32_kernel<DESIGN, Q, WARPS, K><<<grid, G::kThreads, 0, s>>>(a, taps, status_word);
     return cudaGetLastError();
 }
 
 template <int DESIGN>
-cudaError_t launch_conv1d_f32(const Conv1DArgs &a, const float *w, int q, cudaStream_t s, int *launches)
+cudaError_t launch_conv1d_f32(const Conv1DArgs &a, const float *w, int q, unsigned *status_word, cudaStream_t s,
+                              int *launches)
 {
     Taps1D taps;
     for (int k = 0; k < kMaxQ1; ++k) taps.w[k] = k < q ? w[k] : 0.f;
     cudaError_t err = kNoInstantiation;
     switch (q) {
-#define SYSCONV_CASE(QQ) case QQ: err = launch_conv1d_f32_q<DESIGN, QQ>(a, taps, s); break;
+#define SYSCONV_CASE(QQ) case QQ: err = launch_conv1d_f32_q<DESIGN, QQ>(a, taps, status_word, s); break;
         SYSCONV_CASE(1) SYSCONV_CASE(2) SYSCONV_CASE(3) SYSCONV_CASE(4) SYSCONV_CASE(5) SYSCONV_CASE(6)
         SYSCONV_CASE(7) SYSCONV_CASE(8) SYSCONV_CASE(9) SYSCONV_CASE(10) SYSCONV_CASE(11) SYSCONV_CASE(12)
         SYSCONV_CASE(13) SYSCONV_CASE(14) SYSCONV_CASE(15) SYSCONV_CASE(16) SYSCONV_CASE(17) SYSCONV_CASE(18)

@@ -3,9 +3,10 @@
 
 namespace sysconv {
 
-cudaError_t launch_conv1d_f32_os(const Conv1DArgs &a, const float *w, int q, cudaStream_t s, int *launches)
+cudaError_t launch_conv1d_f32_os(const Conv1DArgs &a, const float *w, int q, unsigned *status_word, cudaStream_t s,
+                                 int *launches)
 {
-    return launch_conv1d_f32<SYSCONV_OS>(a, w, q, s, launches);
+    return launch_conv1d_f32<SYSCONV_OS>(a, w, q, status_word, s, launches);
 }
 
 }  // namespace sysconv

@@ -1,12 +1,42 @@
 // C ABI of libsysconv.so: argument validation and dispatch.  See include/sysconv.h
 // for the contract of every entry point.  No device memory is allocated here.
 #include <atomic>
+#include <mutex>
 
 #include "sysconv_common.cuh"
+
+// Raised (set to 1) by a kernel that gave up a bounded wait; read and cleared by sysconv_device_status().
+static __device__ unsigned g_status_word;
 
 namespace {
 
 std::atomic<long long> g_launches{0};
+
+// per-device facts resolved on first use: SM count and the device address of g_status_word
+constexpr int kMaxDevices = 64;
+struct DeviceInfo {
+    bool ready = false;
+    int sm_count = 0;
+    unsigned *status_word = nullptr;
+};
+std::mutex g_device_mutex;
+DeviceInfo g_device[kMaxDevices];
+
+const DeviceInfo *device_info()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(g_device_mutex);
+    DeviceInfo &d = g_device[dev];
+    if (!d.ready) {
+        void *ptr = nullptr;
+        if (cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_status_word) != cudaSuccess || ptr == nullptr) return nullptr;
+        d.status_word = static_cast<unsigned *>(ptr);
+        d.ready = true;
+    }
+    return &d;
+}
 
 inline size_t in_elt_bytes(int dtype) { return dtype == SYSCONV_F32 ? 4 : 1; }
 inline long long align256(long long v) { return (v + 255) & ~255LL; }
@@ -79,9 +109,11 @@ int sysconv1d(const void *x_dev, long long n, long long x_batch_stride, const vo
         a.x_bstride = x_batch_stride; a.y_bstride = y_batch_stride; a.batch = batch;
         const float *w = static_cast<const float *>(w_host);
         int launches = 0;
-        cudaError_t err = design == SYSCONV_OS   ? launch_conv1d_f32_os(a, w, q, s, &launches)
-                          : design == SYSCONV_IS ? launch_conv1d_f32_is(a, w, q, s, &launches)
-                                                 : launch_conv1d_f32_ws(a, w, q, s, &launches);
+        const DeviceInfo *d = device_info();
+        if (!d) return SYSCONV_ECUDA;
+        cudaError_t err = design == SYSCONV_OS   ? launch_conv1d_f32_os(a, w, q, d->status_word, s, &launches)
+                          : design == SYSCONV_IS ? launch_conv1d_f32_is(a, w, q, d->status_word, s, &launches)
+                                                 : launch_conv1d_f32_ws(a, w, q, d->status_word, s, &launches);
         return finish(err, launches);
     }
     // integer signals run as one-row images through the 2-D integer kernels
@@ -204,7 +236,19 @@ const char *sysconv_design_name(int design)
     }
 }
 
-int sysconv_version(void) { return 100; }
+int sysconv_device_status(void)
+{
+    const DeviceInfo *d = device_info();
+    if (!d) return SYSCONV_ECUDA;
+    unsigned flag = 0;
+    if (cudaMemcpy(&flag, d->status_word, sizeof(flag), cudaMemcpyDeviceToHost) != cudaSuccess) return SYSCONV_ECUDA;
+    if (flag == 0) return SYSCONV_OK;
+    flag = 0;
+    if (cudaMemcpy(d->status_word, &flag, sizeof(flag), cudaMemcpyHostToDevice) != cudaSuccess) return SYSCONV_ECUDA;
+    return SYSCONV_ETIMEOUT;
+}
+
+int sysconv_version(void) { return 101; }
 
 long long sysconv_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

@@ -27,14 +27,14 @@ constexpr int R1 = 20;
 constexpr int kWarpIn1 = kLanes * R1;          // 640
 constexpr int kHalo1 = 32;
 constexpr int kWarpOut1 = kWarpIn1 - kHalo1;   // 608
-constexpr int kWarps1 = 8;
-constexpr int kThreads1 = kWarps1 * kLanes;    // 256
-constexpr int kTileOut1 = kWarps1 * kWarpOut1; // 4864 outputs per CTA tile
-constexpr int kTileIn1 = kTileOut1 + kHalo1;   // 4896 inputs per CTA tile
-// weight-stationary arrays inside one warp tile
-constexpr int kWsLanes = 4;                    // lanes per array
-constexpr int kWsArrays = kLanes / kWsLanes;   // 8 arrays per warp
-constexpr int kWsSeg1 = kWarpOut1 / kWsArrays; // 76 outputs per array and tile
+// weight-stationary arrays, 1-D: sixteen two-lane arrays per warp, each streaming a 76-output segment
+// (76 floats = 19 16-byte words: the broadcast reads of a quarter warp fall in distinct banks)
+constexpr int kWsLanes1 = 2;
+constexpr int kWsArrays1 = kLanes / kWsLanes1;  // 16
+constexpr int kWsSeg1 = 76;
+// weight-stationary arrays, 2-D: eight four-lane arrays per warp
+constexpr int kWsLanes = 4;
+constexpr int kWsArrays = kLanes / kWsLanes;    // 8
 
 struct Taps1D {
     float w[kMaxQ1];
@@ -75,9 +75,12 @@ struct Conv2DArgs {
 // Launchers implemented in the per-design translation units.  Each returns a
 // cudaError_t from the launch and adds the number of kernels it launched to
 // *launches.
-cudaError_t launch_conv1d_f32_os(const Conv1DArgs &a, const float *w, int q, cudaStream_t s, int *launches);
-cudaError_t launch_conv1d_f32_is(const Conv1DArgs &a, const float *w, int q, cudaStream_t s, int *launches);
-cudaError_t launch_conv1d_f32_ws(const Conv1DArgs &a, const float *w, int q, cudaStream_t s, int *launches);
+cudaError_t launch_conv1d_f32_os(const Conv1DArgs &a, const float *w, int q, unsigned *status_word, cudaStream_t s,
+                                 int *launches);
+cudaError_t launch_conv1d_f32_is(const Conv1DArgs &a, const float *w, int q, unsigned *status_word, cudaStream_t s,
+                                 int *launches);
+cudaError_t launch_conv1d_f32_ws(const Conv1DArgs &a, const float *w, int q, unsigned *status_word, cudaStream_t s,
+                                 int *launches);
 
 cudaError_t launch_conv2d_f32_os(const Conv2DArgs &a, const float *w, int q, int p, cudaStream_t s, int *launches);
 cudaError_t launch_conv2d_f32_is(const Conv2DArgs &a, const float *w, int q, int p, cudaStream_t s, int *launches);

@@ -105,6 +105,32 @@ def test_1d_unaligned_pointers_and_batch_strides(cuda_device, design, offset):
 
 
 @pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+@pytest.mark.parametrize("q", [1, 4, 13, 16, 32])
+@pytest.mark.parametrize("n_out", [4 * 4864, 4 * 4864 + 1, 7 * 4864 - 1, 100003, 300 * 4864 + 77])
+def test_1d_many_tiles_sizes(cuda_device, design, q, n_out):
+    """Aligned signals of many tiles (bulk-copy staging): whole tiles, ragged last tile, more tiles than
+    CTAs resident at once."""
+    n = n_out + q - 1
+    x, ws = inputs.gen_1d_f32(n, [q], seed=2000 + q)
+    y_ref, s_ref = oracle.conv1d_f32(x, ws[q])
+    assert_close_f32(run_1d(x, ws[q], design, cuda_device), y_ref, s_ref, "n_out=%d q=%d" % (n_out, q))
+    assert B.device_status() == 0
+
+
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+def test_1d_many_tiles_batch(cuda_device, design):
+    # aligned batch strides: the last tile of every signal is ragged and sits in the middle of a CTA's work list
+    rng = np.random.default_rng(9)
+    x = (rng.random((5, 50001), dtype=np.float32) * 2 - 1).astype(np.float32)
+    w = (rng.random(16, dtype=np.float32) * 2 - 1).astype(np.float32)
+    y = run_1d(x, w, design, cuda_device, batch_stride=50004)
+    for b in range(5):
+        y_ref, s_ref = oracle.conv1d_f32(x[b], w)
+        assert_close_f32(y[b], y_ref, s_ref, "batch %d" % b)
+    assert B.device_status() == 0
+
+
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
 def test_1d_exact_on_small_integers(cuda_device, design):
     # integer-valued data: every design must reproduce the sums exactly, whatever its order
     rng = np.random.default_rng(8)
