@@ -3,9 +3,9 @@
 //
 // The PE dimension is the image column c (contiguous in memory); the image row r
 // is the outer loop that the paper leaves untouched (Section 5).  Lane l of a
-// warp holds the R2 = 4 consecutive PEs 4l .. 4l+3 of a 128-PE array; a warp
+// warp holds R consecutive PEs (R = 4 or 8) of a 32R-PE array; a warp
 // marches down a band of rows, loading each input row exactly once into
-// registers with one 128-bit (fp32) or 32-bit (uint8) load per lane.
+// registers with 128-bit (fp32) or 32-bit (uint8) loads (R = 4 or 8 PEs per lane).
 //
 //  * OS / FBS ("multiple FBS 1-D convolutions"): PE c keeps the partial sums of
 //    column c for the P output rows the current input row contributes to.  The
@@ -46,7 +46,7 @@ struct F32Traits {
     static __device__ __forceinline__ acc_t mad(acc_t x, acc_t w, acc_t z) { return fmaf(x, w, z); }
     static __device__ __forceinline__ acc_t mul(acc_t x, acc_t w) { return x * w; }
     // four consecutive elements starting at p (16-byte aligned)
-    static __device__ __forceinline__ void load4v(const in_t *p, acc_t (&v)[4])
+    static __device__ __forceinline__ void load4v(const in_t *p, acc_t *v)
     {
         const float4 t = __ldg(reinterpret_cast<const float4 *>(p));
         v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
@@ -61,7 +61,7 @@ struct U8Traits {
     using taps_t = Taps2DInt;
     static __device__ __forceinline__ acc_t mad(acc_t x, acc_t w, acc_t z) { return x * w + z; }
     static __device__ __forceinline__ acc_t mul(acc_t x, acc_t w) { return x * w; }
-    static __device__ __forceinline__ void load4v(const in_t *p, acc_t (&v)[4])
+    static __device__ __forceinline__ void load4v(const in_t *p, acc_t *v)
     {
         const unsigned t = __ldg(reinterpret_cast<const unsigned *>(p));
         v[0] = t & 0xff; v[1] = (t >> 8) & 0xff; v[2] = (t >> 16) & 0xff; v[3] = t >> 24;
@@ -72,7 +72,7 @@ struct U8Traits {
 // Four consecutive inputs of one row starting at column col; zeros beyond the row's end.
 template <typename Tr>
 __device__ __forceinline__ void load_group(const typename Tr::in_t *__restrict__ rowp, int col, int width,
-                                           bool vec_ok, typename Tr::acc_t (&v)[4])
+                                           bool vec_ok, typename Tr::acc_t *v)
 {
     if (vec_ok && col + 3 < width) {
         Tr::load4v(rowp + col, v);
@@ -85,7 +85,7 @@ __device__ __forceinline__ void load_group(const typename Tr::in_t *__restrict__
 // Four consecutive outputs of one row starting at column col; align = 4, 2 or 1 elements.
 template <typename Tr>
 __device__ __forceinline__ void store_group(typename Tr::out_t *__restrict__ rowp, int col, int col_end,
-                                            int align, const typename Tr::acc_t (&v)[4])
+                                            int align, const typename Tr::acc_t *v)
 {
     using out_t = typename Tr::out_t;
     if (col + 3 < col_end && align == 4) {
@@ -120,18 +120,20 @@ __device__ __forceinline__ int row_alignment(const T *base, long long pitch, lon
 // ---------------------------------------------------------------------------
 // OS / FBS
 // ---------------------------------------------------------------------------
-template <typename Tr, int P, int Q>
-__global__ void __launch_bounds__(kThreads2)
+template <typename Tr, int P, int Q, int R, int MIN_CTAS>
+__global__ void __launch_bounds__(kThreads2, MIN_CTAS)
 conv2d_os_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t taps, const int band_h)
 {
     using in_t = typename Tr::in_t;
     using acc_t = typename Tr::acc_t;
     using out_t = typename Tr::out_t;
+    static_assert(R == 4 || R == 8, "R = PEs per lane");
+    constexpr int kStrip = kLanes * R;          // PEs (= output columns) per strip
     constexpr bool kHalo = Q > 1;
-    constexpr bool kHaloChain = Q - 1 > R2;     // the halo spans more than one lane
+    constexpr bool kHaloChain = Q - 1 > 4;      // the halo spans more than one lane
     const int lane = threadIdx.x & (kLanes - 1);
     const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;
-    const int c0 = strip * kStrip2;
+    const int c0 = strip * kStrip;
     if (c0 >= a.out_w) return;
     const int r0 = blockIdx.y * band_h;
     const int r1 = min(r0 + band_h, a.out_h);
@@ -139,33 +141,37 @@ conv2d_os_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t
     out_t *yb = static_cast<out_t *>(a.y) + blockIdx.z * a.y_bstride;
     const bool x_vec = row_alignment(static_cast<const in_t *>(a.x), a.x_pitch, a.x_bstride, a.batch) == 4;
     const int y_align = row_alignment(static_cast<const out_t *>(a.y), a.y_pitch, a.y_bstride, a.batch);
-    const int col = c0 + R2 * lane;             // first column of this lane's PEs
-    const int hcol = c0 + kStrip2 + R2 * lane;  // halo columns (lanes 0 .. ceil((Q-1)/4)-1)
-    const bool has_halo = kHalo && R2 * lane < Q - 1;
+    const int col = c0 + R * lane;              // first column of this lane's PEs
+    const int hcol = c0 + kStrip + 4 * lane;    // halo columns (lanes 0 .. ceil((Q-1)/4)-1)
+    const bool has_halo = kHalo && 4 * lane < Q - 1;
 
-    acc_t Z[P][R2];
+    acc_t Z[P][R];
 #pragma unroll
     for (int p = 0; p < P; ++p)
 #pragma unroll
-        for (int j = 0; j < R2; ++j) Z[p][j] = 0;
+        for (int j = 0; j < R; ++j) Z[p][j] = 0;
 
-    acc_t nX[R2], nH[R2];
+    acc_t nX[R], nH[4];
 #pragma unroll
-    for (int j = 0; j < R2; ++j) nH[j] = 0;
+    for (int j = 0; j < 4; ++j) nH[j] = 0;
     {
         const in_t *rowp = xb + static_cast<long long>(r0) * a.x_pitch;
-        load_group<Tr>(rowp, col, a.width, x_vec, nX);
+#pragma unroll
+        for (int g = 0; g < R / 4; ++g) load_group<Tr>(rowp, col + 4 * g, a.width, x_vec, &nX[4 * g]);
         if (has_halo) load_group<Tr>(rowp, hcol, a.width, x_vec, nH);
     }
     const int i_end = r1 + P - 1;               // input rows r0 .. i_end-1
 #pragma unroll 1
     for (int i = r0; i < i_end; ++i) {
-        acc_t X[R2], H[R2];
+        acc_t X[R], H[4];
 #pragma unroll
-        for (int j = 0; j < R2; ++j) { X[j] = nX[j]; H[j] = nH[j]; }
+        for (int j = 0; j < R; ++j) X[j] = nX[j];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) H[j] = nH[j];
         if (i + 1 < i_end) {                    // prefetch the next input row
             const in_t *rowp = xb + static_cast<long long>(i + 1) * a.x_pitch;
-            load_group<Tr>(rowp, col, a.width, x_vec, nX);
+#pragma unroll
+            for (int g = 0; g < R / 4; ++g) load_group<Tr>(rowp, col + 4 * g, a.width, x_vec, &nX[4 * g]);
             if (has_halo) load_group<Tr>(rowp, hcol, a.width, x_vec, nH);
         }
         // input row i contributes to output rows i-p through filter row p: one
@@ -177,49 +183,56 @@ conv2d_os_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t
 #pragma unroll
                 for (int p = P - 1; p > 0; --p)
 #pragma unroll
-                    for (int j = 0; j < R2; ++j) Z[p][j] = Tr::mad(X[j], taps.w[p * Q], Z[p - 1][j]);
+                    for (int j = 0; j < R; ++j) Z[p][j] = Tr::mad(X[j], taps.w[p * Q], Z[p - 1][j]);
 #pragma unroll
-                for (int j = 0; j < R2; ++j) Z[0][j] = Tr::mul(X[j], taps.w[0]);
+                for (int j = 0; j < R; ++j) Z[0][j] = Tr::mul(X[j], taps.w[0]);
             } else {
 #pragma unroll
                 for (int p = 0; p < P; ++p)
 #pragma unroll
-                    for (int j = 0; j < R2; ++j) Z[p][j] = Tr::mad(X[j], taps.w[p * Q + q], Z[p][j]);
+                    for (int j = 0; j < R; ++j) Z[p][j] = Tr::mad(X[j], taps.w[p * Q + q], Z[p][j]);
             }
             if (q < Q - 1) {
                 // forward the inputs one PE down; the strip's last PE takes the halo from lane 0
                 const acc_t send = (lane == 0) ? H[0] : X[0];
                 const acc_t in0 = __shfl_sync(kFullMask, send, (lane + 1) & (kLanes - 1));
-                X[0] = X[1]; X[1] = X[2]; X[2] = X[3]; X[3] = in0;
+#pragma unroll
+                for (int j = 0; j < R - 1; ++j) X[j] = X[j + 1];
+                X[R - 1] = in0;
                 acc_t in1 = 0;
                 if (kHaloChain) in1 = __shfl_down_sync(kFullMask, H[0], 1);
                 H[0] = H[1]; H[1] = H[2]; H[2] = H[3]; H[3] = in1;
             }
         }
         const int r = i - (P - 1);              // output row completed by this input row
-        if (r >= r0) store_group<Tr>(yb + static_cast<long long>(r) * a.y_pitch, col, a.out_w, y_align, Z[P - 1]);
+        if (r >= r0) {
+            out_t *orow = yb + static_cast<long long>(r) * a.y_pitch;
+#pragma unroll
+            for (int g = 0; g < R / 4; ++g) store_group<Tr>(orow, col + 4 * g, a.out_w, y_align, &Z[P - 1][4 * g]);
+        }
     }
 }
 
 // ---------------------------------------------------------------------------
 // IS / SBM
 // ---------------------------------------------------------------------------
-template <int Q>
+template <int Q, int R>
 struct IsGeom {
     static constexpr int kDrain = (4 - ((Q - 1) & 3)) & 3;
-    static constexpr int kShift = Q - 1 + kDrain;         // multiple of 4
-    static constexpr int kValid = kStrip2 - kShift;       // outputs per strip
+    static constexpr int kShift = Q - 1 + kDrain;             // multiple of 4
+    static constexpr int kValid = kLanes * R - kShift;        // outputs per strip
 };
 
-template <typename Tr, int P, int Q>
-__global__ void __launch_bounds__(kThreads2)
+template <typename Tr, int P, int Q, int R, int MIN_CTAS>
+__global__ void __launch_bounds__(kThreads2, MIN_CTAS)
 conv2d_is_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t taps, const int band_h)
 {
     using in_t = typename Tr::in_t;
     using acc_t = typename Tr::acc_t;
     using out_t = typename Tr::out_t;
-    constexpr int kShift = IsGeom<Q>::kShift;
-    constexpr int kValid = IsGeom<Q>::kValid;
+    static_assert(R == 4 || R == 8, "R = PEs per lane");
+    constexpr int kShift = IsGeom<Q, R>::kShift;
+    constexpr int kValid = IsGeom<Q, R>::kValid;
     const int lane = threadIdx.x & (kLanes - 1);
     const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;
     const int c0 = strip * kValid;              // first output column = first input column (PE 0)
@@ -230,17 +243,24 @@ conv2d_is_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t
     out_t *yb = static_cast<out_t *>(a.y) + blockIdx.z * a.y_bstride;
     const bool x_vec = row_alignment(static_cast<const in_t *>(a.x), a.x_pitch, a.x_bstride, a.batch) == 4;
     const int y_align = row_alignment(static_cast<const out_t *>(a.y), a.y_pitch, a.y_bstride, a.batch);
-    const int col = c0 + R2 * lane;             // columns held by this lane's PEs
+    const int col = c0 + R * lane;              // columns held by this lane's PEs
     const int ocol = col - kShift;              // output columns its PEs end up holding
     const int oend = min(a.out_w, c0 + kValid);
 
     // PE registers: the P-deep input column of each PE, rows r .. r+P-1
-    acc_t X[P][R2];
+    acc_t X[P][R];
 #pragma unroll
-    for (int p = 0; p < P - 1; ++p)
-        load_group<Tr>(xb + static_cast<long long>(min(r0 + p, a.height - 1)) * a.x_pitch, col, a.width, x_vec, X[p + 1]);
-    acc_t nX[R2];
-    load_group<Tr>(xb + static_cast<long long>(r0 + P - 1) * a.x_pitch, col, a.width, x_vec, nX);
+    for (int p = 0; p < P - 1; ++p) {
+        const in_t *rowp = xb + static_cast<long long>(min(r0 + p, a.height - 1)) * a.x_pitch;
+#pragma unroll
+        for (int g = 0; g < R / 4; ++g) load_group<Tr>(rowp, col + 4 * g, a.width, x_vec, &X[p + 1][4 * g]);
+    }
+    acc_t nX[R];
+    {
+        const in_t *rowp = xb + static_cast<long long>(r0 + P - 1) * a.x_pitch;
+#pragma unroll
+        for (int g = 0; g < R / 4; ++g) load_group<Tr>(rowp, col + 4 * g, a.width, x_vec, &nX[4 * g]);
+    }
 
 #pragma unroll 1
     for (int r = r0; r < r1; ++r) {
@@ -248,120 +268,212 @@ conv2d_is_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t
 #pragma unroll
         for (int p = 0; p < P - 1; ++p)
 #pragma unroll
-            for (int j = 0; j < R2; ++j) X[p][j] = X[p + 1][j];
+            for (int j = 0; j < R; ++j) X[p][j] = X[p + 1][j];
 #pragma unroll
-        for (int j = 0; j < R2; ++j) X[P - 1][j] = nX[j];
-        if (r + 1 < r1)
-            load_group<Tr>(xb + static_cast<long long>(r + P) * a.x_pitch, col, a.width, x_vec, nX);
+        for (int j = 0; j < R; ++j) X[P - 1][j] = nX[j];
+        if (r + 1 < r1) {
+            const in_t *rowp = xb + static_cast<long long>(r + P) * a.x_pitch;
+#pragma unroll
+            for (int g = 0; g < R / 4; ++g) load_group<Tr>(rowp, col + 4 * g, a.width, x_vec, &nX[4 * g]);
+        }
 
-        acc_t Z[R2];
+        acc_t Z[R];
 #pragma unroll
-        for (int q = 0; q < Q + IsGeom<Q>::kDrain; ++q) {
+        for (int q = 0; q < Q + IsGeom<Q, R>::kDrain; ++q) {
             if (q > 0) {
                 // partial sums move one PE up (lane 0 has no left neighbour: invalid PEs)
-                const acc_t up = __shfl_up_sync(kFullMask, Z[R2 - 1], 1);
-                Z[3] = Z[2]; Z[2] = Z[1]; Z[1] = Z[0]; Z[0] = up;
+                const acc_t up = __shfl_up_sync(kFullMask, Z[R - 1], 1);
+#pragma unroll
+                for (int j = R - 1; j > 0; --j) Z[j] = Z[j - 1];
+                Z[0] = up;
             }
             if (q < Q) {
 #pragma unroll
                 for (int p = 0; p < P; ++p)     // t = p + P*q
 #pragma unroll
-                    for (int j = 0; j < R2; ++j)
+                    for (int j = 0; j < R; ++j)
                         Z[j] = (q == 0 && p == 0) ? Tr::mul(X[0][j], taps.w[0])
                                                   : Tr::mad(X[p][j], taps.w[p * Q + q], Z[j]);
             }
         }
-        if (ocol >= c0) store_group<Tr>(yb + static_cast<long long>(r) * a.y_pitch, ocol, oend, y_align, Z);
+        out_t *orow = yb + static_cast<long long>(r) * a.y_pitch;
+#pragma unroll
+        for (int g = 0; g < R / 4; ++g)
+            if (ocol + 4 * g >= c0) store_group<Tr>(orow, ocol + 4 * g, oend, y_align, &Z[4 * g]);
     }
 }
 
 // ---------------------------------------------------------------------------
-// WS (derived from BSM)
+// WS (derived from BSM): PE q keeps the P taps of filter column q; at macro-step T the P+M-1 inputs of
+// image column T that feed the array's M output rows are broadcast to its PEs; every PE adds its P
+// products (sub-steps p = 0..P-1) and the partial sums move one PE up; the last PE emits one output per
+// row and macro-step.
+//
+// An array is four lanes (RW = ceil(Q/4) PEs per lane, unused PEs keep zero taps), a warp holds eight
+// arrays and a CTA 32, stacked over 32*M = 128 output rows.  The CTA streams a segment of the image
+// width through shared memory in chunks of 32 columns, stored TRANSPOSED ([column][row], rows in
+// XOR-swizzled groups of four) so that an array reads the inputs of one image column with 128-bit
+// same-address (broadcast) loads; arrays never refill inside a segment.
 // ---------------------------------------------------------------------------
-constexpr int kWsM2 = 4;                        // output rows per array pass
-constexpr int kWsRows2 = kWsArrays * kWsM2;     // 32 output rows per warp pass
-constexpr int kWsCols2 = 128;                   // output columns streamed per warp pass
+constexpr int kWsM2 = 4;                        // output rows per array
+constexpr int kWsRows2 = kWarps2 * kWsArrays * kWsM2;   // 128 output rows per CTA
+constexpr int kWsChunk = 32;                    // image columns per staged chunk
+constexpr int kWsPitch = 160;                   // rows per staged column (>= 128 + 14 + 2, multiple of 32)
+
+// word index of (column c of the chunk, row) in a staged chunk
+__device__ __forceinline__ int ws_word(int c, int row)
+{
+    return c * kWsPitch + 4 * ((row >> 2) ^ ((c >> 2) & 7)) + (row & 3);
+}
 
 template <typename Tr, int P, int Q>
 __global__ void __launch_bounds__(kThreads2)
-conv2d_ws_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t taps)
+conv2d_ws_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t taps, const int seg_w)
 {
     using in_t = typename Tr::in_t;
     using acc_t = typename Tr::acc_t;
     using out_t = typename Tr::out_t;
     constexpr int RW = (Q + kWsLanes - 1) / kWsLanes;    // PEs per lane
     constexpr int QP = RW * kWsLanes;                    // PEs per array (taps beyond Q are zero)
-    constexpr int K = kWsM2 + P - 1;                     // input rows feeding M output rows
+    constexpr int M = kWsM2;
+    constexpr int K = M + P - 1;                         // input rows feeding M output rows
+    constexpr int KG = (K + 3) / 4;                      // ... in groups of four
+    constexpr int kRowsUsed = kWsRows2 + P - 1;          // staged rows that are ever read
+    __shared__ __align__(16) acc_t s_x[2][kWsChunk * kWsPitch];
+
     const int lane = threadIdx.x & (kLanes - 1);
+    const int warp = threadIdx.x / kLanes;
     const int m_lane = lane & (kWsLanes - 1);
-    const int arr = lane / kWsLanes;
-    const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;
-    const int c0 = strip * kWsCols2;
-    if (c0 >= a.out_w) return;
-    const int r0 = blockIdx.y * kWsRows2 + arr * kWsM2;  // first output row of this array
+    const int arr = warp * kWsArrays + lane / kWsLanes;  // array index inside the CTA, 0..31
+    const int band0 = blockIdx.y * kWsRows2;             // first output row of the CTA
+    const int r0 = band0 + arr * M;                      // first output row of this array
+    const int c0 = blockIdx.x * seg_w;                   // first output column of the segment (multiple of 32)
+    const int c1 = min(c0 + seg_w, a.out_w);             // one past its last output column
     const in_t *xb = static_cast<const in_t *>(a.x) + blockIdx.z * a.x_bstride;
     out_t *yb = static_cast<out_t *>(a.y) + blockIdx.z * a.y_bstride;
+    const bool x_vec = row_alignment(static_cast<const in_t *>(a.x), a.x_pitch, a.x_bstride, a.batch) == 4;
+    const int y_align = row_alignment(static_cast<const out_t *>(a.y), a.y_pitch, a.y_bstride, a.batch);
 
     // PE registers: the P taps of each PE's filter column
     acc_t W[RW][P];
 #pragma unroll
     for (int i = 0; i < RW; ++i) {
-        const int s = m_lane * RW + i;
+        const int sidx = m_lane * RW + i;
 #pragma unroll
-        for (int p = 0; p < P; ++p) W[i][p] = s < Q ? taps.w[p * Q + s] : acc_t(0);
+        for (int p = 0; p < P; ++p) W[i][p] = sidx < Q ? taps.w[p * Q + sidx] : acc_t(0);
     }
-    acc_t Z[kWsM2][RW];
+    acc_t Z[M][RW];
 #pragma unroll
-    for (int m = 0; m < kWsM2; ++m)
+    for (int m = 0; m < M; ++m)
 #pragma unroll
         for (int i = 0; i < RW; ++i) Z[m][i] = 0;
-
-    const in_t *rowp[K];
+    acc_t obuf[M][4];                                    // outputs of four macro-steps, one 128-bit word per row
 #pragma unroll
-    for (int k = 0; k < K; ++k) rowp[k] = xb + static_cast<long long>(min(r0 + k, a.height - 1)) * a.x_pitch;
+    for (int m = 0; m < M; ++m)
+#pragma unroll
+        for (int v = 0; v < 4; ++v) obuf[m][v] = 0;
 
-    const int c_end = min(c0 + kWsCols2, a.out_w);       // output columns [c0, c_end)
-    const int steps = (c_end - c0) + QP - 1;             // macro-steps T = 0 .. steps-1
+    // stage image columns [cc, cc+32) x rows [band0, band0 + kRowsUsed) transposed into buffer `buf`
+    auto stage = [&](int buf, int cc) {
+        acc_t *dst = s_x[buf];
+        for (int idx = threadIdx.x; idx < kRowsUsed * (kWsChunk / 4); idx += kThreads2) {
+            const int row = idx >> 3, i = idx & 7;
+            const in_t *rowp = xb + static_cast<long long>(min(band0 + row, a.height - 1)) * a.x_pitch;
+            acc_t v[4];
+            load_group<Tr>(rowp, cc + 4 * i, a.width, x_vec, v);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) dst[ws_word(4 * i + e, row)] = v[e];
+        }
+    };
+
+    // macro-steps T = 0 .. (c1-c0)+QP-2 produce the segment; up to three more complete the last 128-bit word
+    const int steps = (c1 - c0) + QP - 1 + 3;
+    const int chunks = (steps + kWsChunk - 1) / kWsChunk;
+    stage(0, c0);
+    __syncthreads();
+    const int row_in_cta = arr * M;                      // first staged row this array reads (multiple of 4)
 #pragma unroll 1
-    for (int T = 0; T < steps; ++T) {
-        const int xc = min(c0 + T, a.width - 1);         // image column broadcast at this macro-step
-        acc_t xk[K];
+    for (int j = 0; j < chunks; ++j) {
+        if (j + 1 < chunks) stage((j + 1) & 1, c0 + (j + 1) * kWsChunk);
+        const acc_t *src = s_x[j & 1];
+#pragma unroll 1
+        for (int u = 0; u < kWsChunk / 4; ++u) {
 #pragma unroll
-        for (int k = 0; k < K; ++k) xk[k] = Tr::load1(rowp[k] + xc);
+            for (int v = 0; v < 4; ++v) {
+                const int c = 4 * u + v;                 // column inside the chunk
+                // broadcast: the K inputs of this image column, 128 bits at a time
+                acc_t xk[4 * KG];
 #pragma unroll
-        for (int m = 0; m < kWsM2; ++m) {
-            acc_t up = __shfl_up_sync(kFullMask, Z[m][RW - 1], 1, kWsLanes);
-            if (m_lane == 0) up = 0;                     // PE 0 starts a new sum
-            // sub-step p = 0 also moves the sums one PE up
+                for (int g = 0; g < KG; ++g) {
+                    const int word = c * kWsPitch + 4 * (((row_in_cta >> 2) + g) ^ (u & 7));
+                    if (sizeof(acc_t) == 4) {
+                        const int4 t = *reinterpret_cast<const int4 *>(src + word);
+                        xk[4 * g] = *reinterpret_cast<const acc_t *>(&t.x);
+                        xk[4 * g + 1] = *reinterpret_cast<const acc_t *>(&t.y);
+                        xk[4 * g + 2] = *reinterpret_cast<const acc_t *>(&t.z);
+                        xk[4 * g + 3] = *reinterpret_cast<const acc_t *>(&t.w);
+                    }
+                }
 #pragma unroll
-            for (int i = RW - 1; i > 0; --i) Z[m][i] = Tr::mad(xk[m], W[i][0], Z[m][i - 1]);
-            Z[m][0] = Tr::mad(xk[m], W[0][0], up);
+                for (int m = 0; m < M; ++m) {
+                    acc_t up = __shfl_up_sync(kFullMask, Z[m][RW - 1], 1, kWsLanes);
+                    if (m_lane == 0) up = 0;             // PE 0 starts a new sum
+                    // sub-step p = 0 also moves the sums one PE up
 #pragma unroll
-            for (int p = 1; p < P; ++p)
+                    for (int i = RW - 1; i > 0; --i) Z[m][i] = Tr::mad(xk[m], W[i][0], Z[m][i - 1]);
+                    Z[m][0] = Tr::mad(xk[m], W[0][0], up);
 #pragma unroll
-                for (int i = 0; i < RW; ++i) Z[m][i] = Tr::mad(xk[m + p], W[i][p], Z[m][i]);
+                    for (int p = 1; p < P; ++p)
+#pragma unroll
+                        for (int i = 0; i < RW; ++i) Z[m][i] = Tr::mad(xk[m + p], W[i][p], Z[m][i]);
+                    // the array's last PE now holds output column T-(QP-1); QP is a multiple of 4 and so
+                    // is c0, hence that column is congruent to v+1 modulo 4
+                    obuf[m][(v + 1) & 3] = Z[m][RW - 1];
+                }
+                if (v == 2) {
+                    // columns oc-3 .. oc are complete (oc = T-(QP-1), oc & 3 == 3)
+                    const int oc = c0 + j * kWsChunk + c - (QP - 1);
+                    if (m_lane == kWsLanes - 1 && oc >= c0 + 3 && oc - 3 < c1) {
+#pragma unroll
+                        for (int m = 0; m < M; ++m)
+                            if (r0 + m < a.out_h)
+                                store_group<Tr>(yb + static_cast<long long>(r0 + m) * a.y_pitch, oc - 3, c1, y_align,
+                                                obuf[m]);
+                    }
+                }
+            }
         }
-        const int oc = c0 + T - (QP - 1);                // column completed by the array's last PE
-        if (m_lane == kWsLanes - 1 && oc >= c0) {
-#pragma unroll
-            for (int m = 0; m < kWsM2; ++m)
-                if (r0 + m < a.out_h) yb[static_cast<long long>(r0 + m) * a.y_pitch + oc] = Z[m][RW - 1];
-        }
+        __syncthreads();                                 // chunk j consumed, chunk j+1 staged
     }
 }
 
 // ---------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------
-inline int pick_band_height(int out_h, long long strips_times_batch, int p)
+// Shape of the OS/IS kernels per filter size (measured on B200, 16 x 4096 x 4096 fp32):
+//   small filters are memory-bound: eight PEs per lane and short bands (many CTAs in flight);
+//   mid-size filters: eight PEs per lane under a 128-register cap (four CTAs per SM), which raises the
+//     FMA share of the instruction stream (weight fetches and bookkeeping are per lane and row);
+//   filters with 12 or more rows keep four PEs per lane: P*8 partial sums no longer fit the cap.
+template <typename Tr, int P, int Q>
+struct Shape2D {
+    static constexpr bool kF32 = std::is_same<Tr, F32Traits>::value;
+    static constexpr int kR = (kF32 && P <= 11) ? 8 : 4;
+    static constexpr int kMinCtas = (kF32 && P * Q > 16 && P <= 11) ? 4 : 1;
+};
+
+inline int pick_band_height(int out_h, long long strips_times_batch, int p, int q)
 {
-    const long long target = 148LL * 16;                 // warps wanted in flight
+    // enough CTAs to fill the machine a few times over, bands never shorter than 4*P rows (halo rows
+    // are recomputed per band) nor longer than 256 (64 for the memory-bound small filters)
+    const long long target = 148LL * 16;
     long long bands = (target + strips_times_batch - 1) / strips_times_batch;
     if (bands < 1) bands = 1;
     long long h = (out_h + bands - 1) / bands;
-    const long long lo = p > 8 ? p : 8;
+    const long long lo = 4 * p > 8 ? 4 * p : 8;
+    const long long hi = p * q <= 16 ? 64 : 256;
+    if (h > hi) h = hi;
     if (h < lo) h = lo;
-    if (h > 256) h = 256;
     return static_cast<int>(h);
 }
 
@@ -370,19 +482,30 @@ cudaError_t launch_conv2d_pq(const Conv2DArgs &a, const typename Tr::taps_t &tap
 {
     if (a.batch > 65535) return cudaErrorInvalidConfiguration;
     if (DESIGN == SYSCONV_WS) {
-        const int strips = (a.out_w + kWsCols2 - 1) / kWsCols2;
-        dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + kWsRows2 - 1) / kWsRows2, a.batch);
+        // CTAs = width segments x bands of 128 rows x images; segments are multiples of 32 columns and as
+        // long as possible (each costs QP-1 fill steps) while still giving a few CTAs per SM
+        const long long bands = (a.out_h + kWsRows2 - 1) / kWsRows2;
+        const long long want = 148LL * 6;
+        long long segs = (want + bands * a.batch - 1) / (bands * a.batch);
+        const long long max_segs = (a.out_w + 127) / 128;          // segments of at least 128 columns
+        if (segs > max_segs) segs = max_segs;
+        if (segs < 1) segs = 1;
+        int seg_w = static_cast<int>((a.out_w + segs - 1) / segs);
+        seg_w = (seg_w + kWsChunk - 1) / kWsChunk * kWsChunk;
+        dim3 grid((a.out_w + seg_w - 1) / seg_w, static_cast<unsigned>(bands), a.batch);
         if (grid.y > 65535) return cudaErrorInvalidConfiguration;
-        conv2d_ws_kernel<Tr, P, Q><<<grid, kThreads2, 0, s>>>(a, taps);
-    } else {
-        const int per_strip = DESIGN == SYSCONV_OS ? kStrip2 : IsGeom<Q>::kValid;
-        const int strips = (a.out_w + per_strip - 1) / per_strip;
-        const int band_h = pick_band_height(a.out_h, static_cast<long long>(strips) * a.batch, P);
-        dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + band_h - 1) / band_h, a.batch);
-        if (grid.y > 65535) return cudaErrorInvalidConfiguration;
-        if (DESIGN == SYSCONV_OS) conv2d_os_kernel<Tr, P, Q><<<grid, kThreads2, 0, s>>>(a, taps, band_h);
-        else conv2d_is_kernel<Tr, P, Q><<<grid, kThreads2, 0, s>>>(a, taps, band_h);
+        conv2d_ws_kernel<Tr, P, Q><<<grid, kThreads2, 0, s>>>(a, taps, seg_w);
+        return cudaGetLastError();
     }
+    constexpr int R = Shape2D<Tr, P, Q>::kR;
+    constexpr int MINB = Shape2D<Tr, P, Q>::kMinCtas;
+    const int per_strip = DESIGN == SYSCONV_OS ? kLanes * R : IsGeom<Q, R>::kValid;
+    const int strips = (a.out_w + per_strip - 1) / per_strip;
+    const int band_h = pick_band_height(a.out_h, static_cast<long long>(strips) * a.batch, P, Q);
+    dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + band_h - 1) / band_h, a.batch);
+    if (grid.y > 65535) return cudaErrorInvalidConfiguration;
+    if (DESIGN == SYSCONV_OS) conv2d_os_kernel<Tr, P, Q, R, MINB><<<grid, kThreads2, 0, s>>>(a, taps, band_h);
+    else conv2d_is_kernel<Tr, P, Q, R, MINB><<<grid, kThreads2, 0, s>>>(a, taps, band_h);
     return cudaGetLastError();
 }
 
