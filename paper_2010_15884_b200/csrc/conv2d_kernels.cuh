@@ -120,7 +120,7 @@ __device__ __forceinline__ int row_alignment(const T *base, long long pitch, lon
 // ---------------------------------------------------------------------------
 // OS / FBS
 // ---------------------------------------------------------------------------
-template <typename Tr, int P, int Q, int R, int MIN_CTAS>
+template <typename Tr, int P, int Q, int R, int MIN_CTAS, int PF>
 __global__ void __launch_bounds__(kThreads2, MIN_CTAS)
 conv2d_os_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t taps, const int band_h)
 {
@@ -128,6 +128,7 @@ conv2d_os_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t
     using acc_t = typename Tr::acc_t;
     using out_t = typename Tr::out_t;
     static_assert(R == 4 || R == 8, "R = PEs per lane");
+    static_assert(PF == 1 || PF == 2 || PF == 4, "PF = input rows in flight ahead of the one being processed");
     constexpr int kStrip = kLanes * R;          // PEs (= output columns) per strip
     constexpr bool kHalo = Q > 1;
     constexpr bool kHaloChain = Q - 1 > 4;      // the halo spans more than one lane
@@ -144,6 +145,7 @@ conv2d_os_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t
     const int col = c0 + R * lane;              // first column of this lane's PEs
     const int hcol = c0 + kStrip + 4 * lane;    // halo columns (lanes 0 .. ceil((Q-1)/4)-1)
     const bool has_halo = kHalo && 4 * lane < Q - 1;
+    const int i_end = r1 + P - 1;               // input rows r0 .. i_end-1
 
     acc_t Z[P][R];
 #pragma unroll
@@ -151,29 +153,28 @@ conv2d_os_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t
 #pragma unroll
         for (int j = 0; j < R; ++j) Z[p][j] = 0;
 
-    acc_t nX[R], nH[4];
+    // rows in flight: buffer f holds input row (i + 1 + f) while row i is processed
+    acc_t nX[PF][R], nH[PF][4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) nH[j] = 0;
-    {
-        const in_t *rowp = xb + static_cast<long long>(r0) * a.x_pitch;
+    for (int f = 0; f < PF; ++f)
 #pragma unroll
-        for (int g = 0; g < R / 4; ++g) load_group<Tr>(rowp, col + 4 * g, a.width, x_vec, &nX[4 * g]);
-        if (has_halo) load_group<Tr>(rowp, hcol, a.width, x_vec, nH);
-    }
-    const int i_end = r1 + P - 1;               // input rows r0 .. i_end-1
-#pragma unroll 1
-    for (int i = r0; i < i_end; ++i) {
+        for (int j = 0; j < 4; ++j) nH[f][j] = 0;
+    auto fetch = [&](int row, acc_t *dx, acc_t *dh) {
+        if (row < i_end) {
+            const in_t *rowp = xb + static_cast<long long>(row) * a.x_pitch;
+#pragma unroll
+            for (int g = 0; g < R / 4; ++g) load_group<Tr>(rowp, col + 4 * g, a.width, x_vec, dx + 4 * g);
+            if (has_halo) load_group<Tr>(rowp, hcol, a.width, x_vec, dh);
+        }
+    };
+    // process input row i, whose data sit in buffer f; refill that buffer with row i + PF
+    auto process = [&](int i, int f) {
         acc_t X[R], H[4];
 #pragma unroll
-        for (int j = 0; j < R; ++j) X[j] = nX[j];
+        for (int j = 0; j < R; ++j) X[j] = nX[f][j];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) H[j] = nH[j];
-        if (i + 1 < i_end) {                    // prefetch the next input row
-            const in_t *rowp = xb + static_cast<long long>(i + 1) * a.x_pitch;
-#pragma unroll
-            for (int g = 0; g < R / 4; ++g) load_group<Tr>(rowp, col + 4 * g, a.width, x_vec, &nX[4 * g]);
-            if (has_halo) load_group<Tr>(rowp, hcol, a.width, x_vec, nH);
-        }
+        for (int j = 0; j < 4; ++j) H[j] = nH[f][j];
+        fetch(i + PF, nX[f], nH[f]);
         // input row i contributes to output rows i-p through filter row p: one
         // FBS pass of Q steps, every forwarded input feeding all P rows
 #pragma unroll
@@ -210,6 +211,16 @@ conv2d_os_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t
 #pragma unroll
             for (int g = 0; g < R / 4; ++g) store_group<Tr>(orow, col + 4 * g, a.out_w, y_align, &Z[P - 1][4 * g]);
         }
+    };
+
+#pragma unroll
+    for (int f = 0; f < PF; ++f) fetch(r0 + f, nX[f], nH[f]);
+#pragma unroll 1
+    for (int i = r0; i < i_end; i += PF) {
+        process(i, 0);
+#pragma unroll
+        for (int f = 1; f < PF; ++f)
+            if (i + f < i_end) process(i + f, f);
     }
 }
 
@@ -373,28 +384,44 @@ conv2d_ws_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t
 #pragma unroll
         for (int v = 0; v < 4; ++v) obuf[m][v] = 0;
 
-    // stage image columns [cc, cc+32) x rows [band0, band0 + kRowsUsed) transposed into buffer `buf`
-    auto stage = [&](int buf, int cc) {
-        acc_t *dst = s_x[buf];
-        for (int idx = threadIdx.x; idx < kRowsUsed * (kWsChunk / 4); idx += kThreads2) {
-            const int row = idx >> 3, i = idx & 7;
-            const in_t *rowp = xb + static_cast<long long>(min(band0 + row, a.height - 1)) * a.x_pitch;
-            acc_t v[4];
-            load_group<Tr>(rowp, cc + 4 * i, a.width, x_vec, v);
+    // Staging of image columns [cc, cc+32) x rows [band0, band0 + kRowsUsed): the loads of the next chunk
+    // are issued into registers before the current chunk is processed and written (transposed) after it.
+    constexpr int kStageVec = (kRowsUsed * (kWsChunk / 4) + kThreads2 - 1) / kThreads2;
+    acc_t pf[kStageVec][4];
+    auto stage_load = [&](int cc) {
 #pragma unroll
-            for (int e = 0; e < 4; ++e) dst[ws_word(4 * i + e, row)] = v[e];
+        for (int n = 0; n < kStageVec; ++n) {
+            const int idx = threadIdx.x + n * kThreads2;
+            const int row = idx >> 3, i = idx & 7;
+            if (idx < kRowsUsed * (kWsChunk / 4)) {
+                const in_t *rowp = xb + static_cast<long long>(min(band0 + row, a.height - 1)) * a.x_pitch;
+                load_group<Tr>(rowp, cc + 4 * i, a.width, x_vec, pf[n]);
+            }
+        }
+    };
+    auto stage_store = [&](int buf) {
+        acc_t *dst = s_x[buf];
+#pragma unroll
+        for (int n = 0; n < kStageVec; ++n) {
+            const int idx = threadIdx.x + n * kThreads2;
+            const int row = idx >> 3, i = idx & 7;
+            if (idx < kRowsUsed * (kWsChunk / 4)) {
+#pragma unroll
+                for (int e = 0; e < 4; ++e) dst[ws_word(4 * i + e, row)] = pf[n][e];
+            }
         }
     };
 
     // macro-steps T = 0 .. (c1-c0)+QP-2 produce the segment; up to three more complete the last 128-bit word
     const int steps = (c1 - c0) + QP - 1 + 3;
     const int chunks = (steps + kWsChunk - 1) / kWsChunk;
-    stage(0, c0);
+    stage_load(c0);
+    stage_store(0);
     __syncthreads();
     const int row_in_cta = arr * M;                      // first staged row this array reads (multiple of 4)
 #pragma unroll 1
     for (int j = 0; j < chunks; ++j) {
-        if (j + 1 < chunks) stage((j + 1) & 1, c0 + (j + 1) * kWsChunk);
+        if (j + 1 < chunks) stage_load(c0 + (j + 1) * kWsChunk);
         const acc_t *src = s_x[j & 1];
 #pragma unroll 1
         for (int u = 0; u < kWsChunk / 4; ++u) {
@@ -443,6 +470,7 @@ conv2d_ws_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t
                 }
             }
         }
+        if (j + 1 < chunks) stage_store((j + 1) & 1);    // buffer (j+1)&1 was last read in iteration j-1
         __syncthreads();                                 // chunk j consumed, chunk j+1 staged
     }
 }
@@ -451,30 +479,51 @@ conv2d_ws_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t
 // host side
 // ---------------------------------------------------------------------------
 // Shape of the OS/IS kernels per filter size (measured on B200, 16 x 4096 x 4096 fp32):
-//   small filters are memory-bound: eight PEs per lane and short bands (many CTAs in flight);
-//   mid-size filters: eight PEs per lane under a 128-register cap (four CTAs per SM), which raises the
+//   small filters are memory-bound: eight PEs per lane, short bands (many CTAs in flight) and two input
+//     rows in flight per warp (four measured slower); on small images four PEs per lane instead (twice as many warps);
+//   mid-size OS filters: eight PEs per lane under a 128-register cap (four CTAs per SM), which raises the
 //     FMA share of the instruction stream (weight fetches and bookkeeping are per lane and row);
-//   filters with 12 or more rows keep four PEs per lane: P*8 partial sums no longer fit the cap.
-template <typename Tr, int P, int Q>
+//   OS filters with 12 or more rows, and IS beyond the small filters, keep four PEs per lane: their
+//     P*8 partial sums (OS) or stationary inputs (IS) no longer fit.
+template <typename Tr, int DESIGN, int P, int Q>
 struct Shape2D {
     static constexpr bool kF32 = std::is_same<Tr, F32Traits>::value;
-    static constexpr int kR = (kF32 && P <= 11) ? 8 : 4;
-    static constexpr int kMinCtas = (kF32 && P * Q > 16 && P <= 11) ? 4 : 1;
+    static constexpr bool kSmall = P * Q <= 25;
+    static constexpr int kR = !kF32 ? 4 : kSmall ? 8 : (DESIGN == SYSCONV_OS && P <= 11) ? 8 : 4;
+    static constexpr int kMinCtas = (kF32 && DESIGN == SYSCONV_OS && !kSmall && P <= 11) ? 4 : 1;
+    static constexpr int kPrefetch = kSmall ? 2 : 1;
+    static constexpr bool kAlsoNarrow = kF32 && kSmall;     // a four-PE variant exists for small images
 };
 
 inline int pick_band_height(int out_h, long long strips_times_batch, int p, int q)
 {
-    // enough CTAs to fill the machine a few times over, bands never shorter than 4*P rows (halo rows
-    // are recomputed per band) nor longer than 256 (64 for the memory-bound small filters)
+    // enough CTAs to fill the machine a few times over; bands never shorter than 2*P rows (halo rows are
+    // recomputed per band) nor longer than 256 (64 for the memory-bound small filters)
     const long long target = 148LL * 16;
     long long bands = (target + strips_times_batch - 1) / strips_times_batch;
     if (bands < 1) bands = 1;
     long long h = (out_h + bands - 1) / bands;
-    const long long lo = 4 * p > 8 ? 4 * p : 8;
-    const long long hi = p * q <= 16 ? 64 : 256;
+    const long long lo = 2 * p > 8 ? 2 * p : 8;
+    const long long hi = p * q <= 25 ? 64 : 256;
     if (h > hi) h = hi;
     if (h < lo) h = lo;
     return static_cast<int>(h);
+}
+
+template <typename Tr, int DESIGN, int P, int Q, int R>
+cudaError_t launch_conv2d_osis(const Conv2DArgs &a, const typename Tr::taps_t &taps, cudaStream_t s)
+{
+    using Sh = Shape2D<Tr, DESIGN, P, Q>;
+    const int per_strip = DESIGN == SYSCONV_OS ? kLanes * R : IsGeom<Q, R>::kValid;
+    const int strips = (a.out_w + per_strip - 1) / per_strip;
+    const int band_h = pick_band_height(a.out_h, static_cast<long long>(strips) * a.batch, P, Q);
+    dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + band_h - 1) / band_h, a.batch);
+    if (grid.y > 65535) return cudaErrorInvalidConfiguration;
+    if (DESIGN == SYSCONV_OS)
+        conv2d_os_kernel<Tr, P, Q, R, Sh::kMinCtas, Sh::kPrefetch><<<grid, kThreads2, 0, s>>>(a, taps, band_h);
+    else
+        conv2d_is_kernel<Tr, P, Q, R, Sh::kMinCtas><<<grid, kThreads2, 0, s>>>(a, taps, band_h);
+    return cudaGetLastError();
 }
 
 template <typename Tr, int DESIGN, int P, int Q>
@@ -497,16 +546,15 @@ cudaError_t launch_conv2d_pq(const Conv2DArgs &a, const typename Tr::taps_t &tap
         conv2d_ws_kernel<Tr, P, Q><<<grid, kThreads2, 0, s>>>(a, taps, seg_w);
         return cudaGetLastError();
     }
-    constexpr int R = Shape2D<Tr, P, Q>::kR;
-    constexpr int MINB = Shape2D<Tr, P, Q>::kMinCtas;
-    const int per_strip = DESIGN == SYSCONV_OS ? kLanes * R : IsGeom<Q, R>::kValid;
-    const int strips = (a.out_w + per_strip - 1) / per_strip;
-    const int band_h = pick_band_height(a.out_h, static_cast<long long>(strips) * a.batch, P, Q);
-    dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + band_h - 1) / band_h, a.batch);
-    if (grid.y > 65535) return cudaErrorInvalidConfiguration;
-    if (DESIGN == SYSCONV_OS) conv2d_os_kernel<Tr, P, Q, R, MINB><<<grid, kThreads2, 0, s>>>(a, taps, band_h);
-    else conv2d_is_kernel<Tr, P, Q, R, MINB><<<grid, kThreads2, 0, s>>>(a, taps, band_h);
-    return cudaGetLastError();
+    using Sh = Shape2D<Tr, DESIGN, P, Q>;
+    if (Sh::kAlsoNarrow) {
+        // small image: with eight PEs per lane there would be fewer than ~8 warps per SM even with the
+        // shortest bands, so take four PEs per lane
+        const long long strips8 = (a.out_w + 255) / 256;
+        const long long warps8 = strips8 * a.batch * ((a.out_h + 7) / 8);
+        if (warps8 < 148LL * 8 * 4) return launch_conv2d_osis<Tr, DESIGN, P, Q, 4>(a, taps, s);
+    }
+    return launch_conv2d_osis<Tr, DESIGN, P, Q, Sh::kR>(a, taps, s);
 }
 
 template <typename Tr, int DESIGN, int P>
