@@ -33,7 +33,10 @@
  *     copied by value into the launch, so it may be freed or changed as soon as
  *     the call returns.
  *   - Ownership: the caller owns every buffer.  The library allocates no
- *     device memory and keeps no state between calls except a launch counter.
+ *     device memory.  State kept between calls: a launch counter, one status
+ *     word in device memory per GPU (see sysconv_device_status) and, after the
+ *     first pipelined host-buffer call on a GPU, two helper streams and a few
+ *     events for that GPU.
  *   - Asynchrony: the work is enqueued on `stream` (a cudaStream_t passed as
  *     void*, NULL = the default stream); the call does not synchronise.
  *   - x and y must not overlap.
@@ -102,10 +105,16 @@ int sysconv2d(const void *x_dev, int width, int height, long long x_pitch, long 
 /*
  * The same two operations for callers whose data lives in HOST memory
  * (densely packed: pitch = row length, batch stride = array size).  The call
- * enqueues, on `stream`: the host-to-device copy of x into the caller's device
- * workspace, the kernel, and the device-to-host copy of y; it does not
- * synchronise (synchronise the stream before reading y_host).  Copies overlap
- * only if the host buffers are page-locked.
+ * enqueues the host-to-device copy of x into the caller's device workspace,
+ * the kernel(s), and the device-to-host copy of y, ordered after the work
+ * already in `stream` and before work enqueued in `stream` later; it does not
+ * synchronise (synchronise the stream before reading y_host).  Large problems
+ * (a long single signal, several images, a large single image) are cut into up
+ * to 16 chunks whose copy in, kernel and copy out overlap on two helper
+ * streams of the library (the kernels run on `stream`); this needs page-locked
+ * host buffers to be effective.  sysconv1d_host_plain is the unchunked form:
+ * one copy in, one kernel, one copy out, everything on `stream`, no helper
+ * streams or events.
  *   workspace_dev / workspace_bytes   DEVICE scratch owned by the caller, at
  *       least sysconv*_host_workspace_bytes(...) bytes, 256-byte aligned.
  * Returns SYSCONV_EINVAL if the workspace is too small.
@@ -116,6 +125,10 @@ long long sysconv2d_host_workspace_bytes(int width, int height, int q, int p, in
 int sysconv1d_host(const void *x_host, long long n, const void *w_host, int q,
                    void *y_host, int batch, int dtype, int design,
                    void *workspace_dev, long long workspace_bytes, void *stream);
+
+int sysconv1d_host_plain(const void *x_host, long long n, const void *w_host, int q,
+                         void *y_host, int batch, int dtype, int design,
+                         void *workspace_dev, long long workspace_bytes, void *stream);
 
 int sysconv2d_host(const void *x_host, int width, int height, const void *w_host, int q, int p,
                    void *y_host, int batch, int dtype, int design,
@@ -133,8 +146,9 @@ int sysconv2d_host(const void *x_host, int width, int height, const void *w_host
  *
  * This entry point takes the same host buffers and stages them in a fixed array
  * that is part of the library's device image, so it allocates nothing: no
- * cudaMalloc/cudaFree, no allocating library call.  Same arguments and results as
- * sysconv1d_host, minus the workspace.
+ * cudaMalloc/cudaFree, no allocating library call (it runs the plain sequence of
+ * sysconv1d_host_plain, so it creates no streams or events either).  Same
+ * arguments and results as sysconv1d_host, minus the workspace.
  *   - Limit: sysconv1d_host_workspace_bytes(n, q, batch, dtype) must not exceed
  *     sysconv_static_scratch_bytes() (16 MiB: about 2 Mi fp32 samples in one
  *     signal, or the same total over a batch).  Larger problems return

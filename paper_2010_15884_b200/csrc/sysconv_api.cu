@@ -49,6 +49,50 @@ int finish(cudaError_t err, int launches)
     return SYSCONV_OK;
 }
 
+// Helper streams and events of the pipelined host-buffer entry points: one set per device, created on
+// first use and kept for the life of the process.  Copies in run on `h2d`, copies out on `d2h`, kernels
+// on the caller's stream; fork/join events tie the helpers into the caller's stream order.
+constexpr int kMaxPipeChunks = 16;
+struct HostPipe {
+    bool ready = false;
+    std::mutex busy;                            // one pipelined call at a time per device
+    cudaStream_t h2d = nullptr, d2h = nullptr;
+    cudaEvent_t forked = nullptr, joined = nullptr;
+    cudaEvent_t in_done[kMaxPipeChunks], k_done[kMaxPipeChunks];
+    bool fork(cudaStream_t s)
+    {
+        return cudaEventRecord(forked, s) == cudaSuccess && cudaStreamWaitEvent(h2d, forked, 0) == cudaSuccess &&
+               cudaStreamWaitEvent(d2h, forked, 0) == cudaSuccess;
+    }
+    bool join(cudaStream_t s)
+    {
+        bool ok = cudaEventRecord(joined, d2h) == cudaSuccess && cudaStreamWaitEvent(s, joined, 0) == cudaSuccess;
+        ok = ok && cudaEventRecord(joined, h2d) == cudaSuccess && cudaStreamWaitEvent(s, joined, 0) == cudaSuccess;
+        return ok;
+    }
+};
+HostPipe g_pipe[kMaxDevices];
+
+HostPipe *host_pipe()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(g_device_mutex);
+    HostPipe &p = g_pipe[dev];
+    if (!p.ready) {
+        bool ok = cudaStreamCreateWithFlags(&p.h2d, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaStreamCreateWithFlags(&p.d2h, cudaStreamNonBlocking) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&p.forked, cudaEventDisableTiming) == cudaSuccess &&
+                  cudaEventCreateWithFlags(&p.joined, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; ok && i < kMaxPipeChunks; ++i)
+            ok = cudaEventCreateWithFlags(&p.in_done[i], cudaEventDisableTiming) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&p.k_done[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) return nullptr;
+        p.ready = true;
+    }
+    return &p;
+}
+
 bool valid_enums(int dtype, int design)
 {
     return (dtype == SYSCONV_F32 || dtype == SYSCONV_U8S8_S32) &&
@@ -171,8 +215,10 @@ long long sysconv2d_host_workspace_bytes(int width, int height, int q, int p, in
     return align256(in) + align256(out);
 }
 
-int sysconv1d_host(const void *x_host, long long n, const void *w_host, int q, void *y_host, int batch,
-                   int dtype, int design, void *workspace_dev, long long workspace_bytes, void *stream)
+// ---- host-buffer entry points --------------------------------------------------------------------
+// Plain form: one copy in, the kernel, one copy out, all on the caller's stream.
+int sysconv1d_host_plain(const void *x_host, long long n, const void *w_host, int q, void *y_host, int batch,
+                         int dtype, int design, void *workspace_dev, long long workspace_bytes, void *stream)
 {
     if (!x_host || !y_host || !w_host || !workspace_dev) return SYSCONV_EINVAL;
     const long long need = sysconv1d_host_workspace_bytes(n, q, batch, dtype);
@@ -190,6 +236,51 @@ int sysconv1d_host(const void *x_host, long long n, const void *w_host, int q, v
     return SYSCONV_OK;
 }
 
+int sysconv1d_host(const void *x_host, long long n, const void *w_host, int q, void *y_host, int batch,
+                   int dtype, int design, void *workspace_dev, long long workspace_bytes, void *stream)
+{
+    if (!x_host || !y_host || !w_host || !workspace_dev) return SYSCONV_EINVAL;
+    const long long need = sysconv1d_host_workspace_bytes(n, q, batch, dtype);
+    if (need < 0 || workspace_bytes < need) return SYSCONV_EINVAL;
+    if ((reinterpret_cast<unsigned long long>(workspace_dev) & 255ull) != 0) return SYSCONV_EINVAL;
+    const long long n_out = n - q + 1;
+    // long single signals: cut into chunks so that the copy in of chunk c+1, the kernel of chunk c and
+    // the copy out of chunk c-1 overlap (PCIe is full duplex)
+    const long long kChunkMin = 1LL << 20;
+    long long chunks = (batch == 1) ? n_out / kChunkMin : 1;
+    if (chunks > kMaxPipeChunks) chunks = kMaxPipeChunks;
+    if (chunks < 2)
+        return sysconv1d_host_plain(x_host, n, w_host, q, y_host, batch, dtype, design, workspace_dev,
+                                    workspace_bytes, stream);
+    HostPipe *pipe = host_pipe();
+    if (!pipe) return SYSCONV_ECUDA;
+    std::lock_guard<std::mutex> lock(pipe->busy);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const long long esz = (long long)in_elt_bytes(dtype);
+    char *xd = static_cast<char *>(workspace_dev);
+    char *yd = xd + align256(n * esz);
+    long long len = (n_out + chunks - 1) / chunks;
+    len = (len + 9727) / 9728 * 9728;                    // whole tiles of every design; keeps 16-byte alignment
+    if (!pipe->fork(s)) return SYSCONV_ECUDA;
+    int c = 0;
+    for (long long o0 = 0; o0 < n_out; o0 += len, ++c) {
+        const long long o1 = o0 + len < n_out ? o0 + len : n_out;
+        const long long in0 = o0 == 0 ? 0 : o0 + q - 1;           // inputs not yet copied by earlier chunks
+        const long long in1 = o1 + q - 1;
+        if (cudaMemcpyAsync(xd + in0 * esz, static_cast<const char *>(x_host) + in0 * esz, (in1 - in0) * esz,
+                            cudaMemcpyHostToDevice, pipe->h2d) != cudaSuccess) return SYSCONV_ECUDA;
+        if (cudaEventRecord(pipe->in_done[c], pipe->h2d) != cudaSuccess) return SYSCONV_ECUDA;
+        if (cudaStreamWaitEvent(s, pipe->in_done[c], 0) != cudaSuccess) return SYSCONV_ECUDA;
+        const int st = sysconv1d(xd + o0 * esz, (o1 - o0) + q - 1, 0, w_host, q, yd + o0 * 4, 0, 1, dtype, design, stream);
+        if (st != SYSCONV_OK) { pipe->join(s); return st; }
+        if (cudaEventRecord(pipe->k_done[c], s) != cudaSuccess) return SYSCONV_ECUDA;
+        if (cudaStreamWaitEvent(pipe->d2h, pipe->k_done[c], 0) != cudaSuccess) return SYSCONV_ECUDA;
+        if (cudaMemcpyAsync(static_cast<char *>(y_host) + o0 * 4, yd + o0 * 4, (o1 - o0) * 4,
+                            cudaMemcpyDeviceToHost, pipe->d2h) != cudaSuccess) return SYSCONV_ECUDA;
+    }
+    return pipe->join(s) ? SYSCONV_OK : SYSCONV_ECUDA;
+}
+
 int sysconv2d_host(const void *x_host, int width, int height, const void *w_host, int q, int p, void *y_host,
                    int batch, int dtype, int design, void *workspace_dev, long long workspace_bytes,
                    void *stream)
@@ -199,18 +290,58 @@ int sysconv2d_host(const void *x_host, int width, int height, const void *w_host
     if (need < 0 || workspace_bytes < need) return SYSCONV_EINVAL;
     if ((reinterpret_cast<unsigned long long>(workspace_dev) & 255ull) != 0) return SYSCONV_EINVAL;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const long long esz = (long long)in_elt_bytes(dtype);
+    const int out_w = width - q + 1, out_h = height - p + 1;
     const long long x_img = (long long)width * height;
-    const long long y_img = (long long)(width - q + 1) * (height - p + 1);
-    const long long x_bytes = x_img * batch * (long long)in_elt_bytes(dtype);
-    const long long y_bytes = y_img * batch * 4LL;
+    const long long y_img = (long long)out_w * out_h;
     char *xd = static_cast<char *>(workspace_dev);
-    char *yd = xd + align256(x_bytes);
-    if (cudaMemcpyAsync(xd, x_host, x_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) return SYSCONV_ECUDA;
-    const int st = sysconv2d(xd, width, height, width, x_img, w_host, q, p, yd, width - q + 1, y_img, batch,
-                             dtype, design, stream);
-    if (st != SYSCONV_OK) return st;
-    if (cudaMemcpyAsync(y_host, yd, y_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SYSCONV_ECUDA;
-    return SYSCONV_OK;
+    char *yd = xd + align256(x_img * batch * esz);
+
+    // chunks: whole images when there are several, else bands of output rows of a large image
+    const bool by_image = batch >= 2;
+    long long chunks = by_image ? batch : y_img / (1LL << 20);
+    if (chunks > kMaxPipeChunks) chunks = kMaxPipeChunks;
+    if (chunks < 2) {
+        if (cudaMemcpyAsync(xd, x_host, x_img * batch * esz, cudaMemcpyHostToDevice, s) != cudaSuccess) return SYSCONV_ECUDA;
+        const int st = sysconv2d(xd, width, height, width, x_img, w_host, q, p, yd, out_w, y_img, batch, dtype, design, stream);
+        if (st != SYSCONV_OK) return st;
+        if (cudaMemcpyAsync(y_host, yd, y_img * batch * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SYSCONV_ECUDA;
+        return SYSCONV_OK;
+    }
+    HostPipe *pipe = host_pipe();
+    if (!pipe) return SYSCONV_ECUDA;
+    std::lock_guard<std::mutex> lock(pipe->busy);
+    if (!pipe->fork(s)) return SYSCONV_ECUDA;
+    const long long unit = by_image ? batch : out_h;             // images, or output rows of the one image
+    const long long per = (unit + chunks - 1) / chunks;
+    int c = 0;
+    for (long long u0 = 0; u0 < unit; u0 += per, ++c) {
+        const long long u1 = u0 + per < unit ? u0 + per : unit;
+        long long in_off, in_len, y_off, y_len;
+        int st;
+        if (by_image) {
+            in_off = u0 * x_img; in_len = (u1 - u0) * x_img; y_off = u0 * y_img; y_len = (u1 - u0) * y_img;
+        } else {
+            const long long row0 = u0 == 0 ? 0 : u0 + p - 1;     // input rows not yet copied by earlier chunks
+            in_off = row0 * width; in_len = (u1 + p - 1 - row0) * width; y_off = u0 * out_w; y_len = (u1 - u0) * out_w;
+        }
+        if (cudaMemcpyAsync(xd + in_off * esz, static_cast<const char *>(x_host) + in_off * esz, in_len * esz,
+                            cudaMemcpyHostToDevice, pipe->h2d) != cudaSuccess) return SYSCONV_ECUDA;
+        if (cudaEventRecord(pipe->in_done[c], pipe->h2d) != cudaSuccess) return SYSCONV_ECUDA;
+        if (cudaStreamWaitEvent(s, pipe->in_done[c], 0) != cudaSuccess) return SYSCONV_ECUDA;
+        if (by_image)
+            st = sysconv2d(xd + u0 * x_img * esz, width, height, width, x_img, w_host, q, p, yd + u0 * y_img * 4, out_w,
+                           y_img, static_cast<int>(u1 - u0), dtype, design, stream);
+        else
+            st = sysconv2d(xd + u0 * width * esz, width, static_cast<int>(u1 - u0) + p - 1, width, 0, w_host, q, p,
+                           yd + u0 * out_w * 4, out_w, 0, 1, dtype, design, stream);
+        if (st != SYSCONV_OK) { pipe->join(s); return st; }
+        if (cudaEventRecord(pipe->k_done[c], s) != cudaSuccess) return SYSCONV_ECUDA;
+        if (cudaStreamWaitEvent(pipe->d2h, pipe->k_done[c], 0) != cudaSuccess) return SYSCONV_ECUDA;
+        if (cudaMemcpyAsync(static_cast<char *>(y_host) + y_off * 4, yd + y_off * 4, y_len * 4, cudaMemcpyDeviceToHost,
+                            pipe->d2h) != cudaSuccess) return SYSCONV_ECUDA;
+    }
+    return pipe->join(s) ? SYSCONV_OK : SYSCONV_ECUDA;
 }
 
 const char *sysconv_status_string(int status)

@@ -13,6 +13,11 @@
 
 #include "sysconv_common.cuh"
 
+// plain host-buffer sequence, defined beside sysconv1d_host
+extern "C" int sysconv1d_host_plain(const void *x_host, long long n, const void *w_host, int q, void *y_host,
+                                    int batch, int dtype, int design, void *workspace_dev,
+                                    long long workspace_bytes, void *stream);
+
 namespace {
 
 constexpr long long kStaticScratchBytes = 16LL << 20;     // 16 MiB: x and y of up to ~2 Mi fp32 samples
@@ -58,11 +63,11 @@ int sysconv1d_host_static(const void *x_host, long long n, const void *w_host, i
     void *scratch = nullptr;
     const int st = static_scratch(&scratch);
     if (st != SYSCONV_OK) return st;
-    // Same sequence as sysconv1d_host, with the built-in staging area as the workspace: copy in,
-    // convolve, copy out, all on `stream`.  The kernels read x only inside [0, n) and write every
+    // The plain sequence of sysconv1d_host (no helper streams or events are created), with the built-in
+    // staging area as the workspace: copy in, convolve, copy out, all on `stream`.  The kernels read x only inside [0, n) and write every
     // one of the n-q+1 outputs, so stale contents of the area from earlier calls are never seen.
-    return sysconv1d_host(x_host, n, w_host, q, y_host, batch, dtype, design, scratch, kStaticScratchBytes,
-                          stream);
+    return sysconv1d_host_plain(x_host, n, w_host, q, y_host, batch, dtype, design, scratch, kStaticScratchBytes,
+                                stream);
 }
 
 }  // extern "C"

@@ -334,6 +334,32 @@ def test_host_entry_points(cuda_device, design):
         np.testing.assert_array_equal(yh2[b].numpy(), oracle.conv2d_u8s8_s32(x2[b], ws2[(3, 3)]))
 
 
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+def test_host_entry_points_chunked_overlap(cuda_device, design):
+    """Problems large enough for the chunked (copy/compute overlapped) form of the host-buffer calls."""
+    n, q = 5_000_003, 16
+    x, ws = inputs.gen_1d_f32(n, [q], seed=31)
+    xh = torch.from_numpy(x).pin_memory()
+    yh = torch.full((n - q + 1,), float("nan"), dtype=torch.float32).pin_memory()
+    work = torch.empty(B.host_workspace_bytes((n,), (q,)), dtype=torch.uint8, device=cuda_device)
+    B.sysconv1d_host(xh, ws[q], yh, design, work)
+    torch.cuda.synchronize()
+    y_ref, s_ref = oracle.conv1d_f32(x, ws[q])
+    assert_close_f32(yh.numpy(), y_ref, s_ref, "1-D host, chunked")
+
+    # one large image: bands of rows; three images: one chunk per image
+    for shape in ((1, 1500, 1400), (3, 300, 500)):
+        x2, ws2 = inputs.gen_2d_f32(shape[2], shape[1], [(5, 3)], seed=32, batch=shape[0])
+        xh2 = torch.from_numpy(x2).pin_memory()
+        yh2 = torch.full((shape[0], shape[1] - 4, shape[2] - 2), float("nan"), dtype=torch.float32).pin_memory()
+        work2 = torch.empty(B.host_workspace_bytes(shape, (5, 3)), dtype=torch.uint8, device=cuda_device)
+        B.sysconv2d_host(xh2, ws2[(5, 3)], yh2, design, work2)
+        torch.cuda.synchronize()
+        for b in range(shape[0]):
+            y_ref, s_ref = oracle.conv2d_f32(x2[b], ws2[(5, 3)])
+            assert_close_f32(yh2[b].numpy(), y_ref, s_ref, "2-D host, chunked %s image %d" % (shape, b))
+
+
 def test_unsupported_and_invalid_on_device(cuda_device):
     x = torch.zeros(1000, device=cuda_device)
     with pytest.raises(B.SysconvError) as e:
