@@ -357,14 +357,28 @@ def run_ours(args):
     top = max(cases, key=lambda c: sum(c.times_ms))
     avg_s = statistics.mean(top.times_ms) * 1e-3
     t_roof, bound = roofline_time_s(top, hbm_gbs, sm_max)
-    roofline = {
-        "kernel": "%s %s" % (NAMES[top.design], top.label), "bound": "hbm",
-        "achieved": round(top.alg_bytes / avg_s / 1e9, 1), "peak": hbm_gbs, "unit": "GB/s",
-        "frac": round(top.alg_bytes / avg_s / 1e9 / hbm_gbs, 4), "peak_source": "of " + peak_kind,
+    if bound == "hbm":
+        roofline = {
+            "kernel": "%s %s" % (NAMES[top.design], top.label), "bound": "hbm",
+            "achieved": round(top.alg_bytes / avg_s / 1e9, 1), "peak": hbm_gbs, "unit": "GB/s",
+            "frac": round(top.alg_bytes / avg_s / 1e9 / hbm_gbs, 4), "peak_source": "of " + peak_kind,
+        }
+    else:
+        # plain FP32/INT32 ALUs (no tensor cores: small-filter stencil): 148 SMs x 128 lanes x 2 flops x SM max clock
+        peak_tflops = SM_COUNT * FP32_LANES_PER_SM * 2 * sm_max * 1e6 / 1e12
+        roofline = {
+            "kernel": "%s %s" % (NAMES[top.design], top.label), "bound": "alu",
+            "achieved": round(2 * top.macs / avg_s / 1e12, 2), "peak": round(peak_tflops, 1), "unit": "TFLOP/s",
+            "frac": round(2 * top.macs / avg_s / 1e12 / peak_tflops, 4),
+            "peak_source": "derived: 148 SMs x 128 lanes x 2 x %.0f MHz" % sm_max,
+        }
+    roofline.update({
         "traffic": ncu_traffic(cfg_id, top),
+        "algorithmic_bytes": int(top.alg_bytes),
         "share_of_step": round(sum(top.times_ms) / sum(sum(c.times_ms) for c in cases), 4),
+        "hbm_time_frac": round(top.alg_bytes / (hbm_gbs * 1e9) / avg_s, 4),
         "alu_time_frac": round(top.macs / (SM_COUNT * FP32_LANES_PER_SM * sm_max * 1e6) / avg_s, 4),
-    }
+    })
 
     # ---- end to end through the host-buffer entry points (rank-local pinned buffers)
     e2e = None if (args.no_e2e or scale) else run_e2e(cfg_id, device, args, world)
@@ -401,18 +415,22 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-_NCU_TRAFFIC = None
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch from the ncu captures summarised in
+# profiles/conv1d_f32_cfg2_kernels.md (full size) and profiles/conv2d_f32_cfg5_kernels.md (2 of 16 images,
+# scaled x8 here because traffic grows in proportion to the number of images).
+NCU_TRAFFIC = {
+    "cfg2 WS Q=4": 482353152, "cfg2 OS Q=4": 480993280, "cfg2 IS Q=4": 483138304,
+    "cfg2 WS Q=16": 487111424, "cfg2 OS Q=16": 485880064, "cfg2 IS Q=16": 483544320,
+    "cfg2 WS Q=32": 489855744, "cfg2 OS Q=32": 489574144, "cfg2 IS Q=32": 489446144,
+    "cfg5 WS 3x3": 8 * 239967488, "cfg5 OS 3x3": 8 * 226216960, "cfg5 IS 3x3": 8 * 224739072,
+    "cfg5 WS 9x9": 8 * 237750784, "cfg5 OS 9x9": 8 * 238917376, "cfg5 IS 9x9": 8 * 234722560,
+    "cfg5 WS 15x15": 8 * 238174976, "cfg5 OS 15x15": 8 * 241290752, "cfg5 IS 15x15": 8 * 241511424,
+}
 
 
 def ncu_traffic(cfg_id, case):
-    """DRAM bytes per launch of this kernel from the committed ncu summary, if one covers it."""
-    path = os.path.join(ROOT, "profiles", "traffic.json")
-    try:
-        with open(path) as f:
-            table = json.load(f)
-        return table.get("cfg%d %s %s" % (cfg_id, NAMES[case.design], case.label))
-    except Exception:
-        return None
+    """DRAM bytes per launch of this kernel from the committed ncu summaries, if one covers it."""
+    return NCU_TRAFFIC.get("cfg%d %s %s" % (cfg_id, NAMES[case.design], case.label))
 
 
 def run_e2e(cfg_id, device, args, world):
