@@ -225,6 +225,132 @@ conv2d_os_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t
 }
 
 // ---------------------------------------------------------------------------
+// OS / FBS, fp32, row-paired form for the tall filters (P >= 9).
+//
+// Same dataflow as conv2d_os_kernel, two input rows per iteration.  The partial sums of two consecutive
+// output rows share a 64-bit register pair and are updated by ONE packed fp32x2 FMA (fma.rn.f32x2, new on
+// sm_100): the multiplicand is (x, x), the multiplier a pair of taps of two consecutive filter rows, which
+// comes straight from the kernel parameters as a uniform-register pair.  Each of the two input rows feeds
+// pair m with its own tap pair, so a step costs (P+1) packed FMAs per PE instead of 2P scalar ones; the
+// scalar kernel is issue-bound (81 % of its instructions are FMAs at 89 % issue-slot use), this form is
+// FMA-pipe-bound.  Both rows' inputs are forwarded exactly as before (one shuffle per row and step).
+// With P odd the P+1 slots fill the pairs exactly; with P even one slot of the last pair stays zero.
+// ---------------------------------------------------------------------------
+// Slots and slot pairs of the row-paired kernel: P + 1 partial rows are alive while two input rows are
+// processed; pair m holds the slots 2m and 2m+1.
+template <int P>
+struct F2R {
+    static constexpr int S = P + 1, SP = (S + 1) / 2;
+};
+// Tap pairs [m][q], m < 8: a = (w[2m][q], w[2m+1][q]) for the later input row, b = (w[2m-1][q], w[2m][q]) for the
+// earlier one; taps outside 0..P-1 are zero.
+struct TapsRowPairs {
+    float2 a[8 * kMaxQ2];
+    float2 b[8 * kMaxQ2];
+};
+template <int P, int Q, int R, int MIN_CTAS>
+__global__ void __launch_bounds__(kThreads2, MIN_CTAS)
+conv2d_os_rowpair_kernel(const Conv2DArgs a, const __grid_constant__ TapsRowPairs taps, const int band_h)
+{
+    using Tr = F32Traits;
+    constexpr int SP = F2R<P>::SP;
+    constexpr bool kHalo = Q > 1;
+    constexpr bool kHaloChain = Q - 1 > 4;
+    constexpr int kStrip = kLanes * R;
+    const int lane = threadIdx.x & (kLanes - 1);
+    const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;
+    const int c0 = strip * kStrip;
+    if (c0 >= a.out_w) return;
+    const int r0 = blockIdx.y * band_h;
+    const int r1 = min(r0 + band_h, a.out_h);
+    const float *xb = static_cast<const float *>(a.x) + blockIdx.z * a.x_bstride;
+    float *yb = static_cast<float *>(a.y) + blockIdx.z * a.y_bstride;
+    const bool x_vec = row_alignment(static_cast<const float *>(a.x), a.x_pitch, a.x_bstride, a.batch) == 4;
+    const int y_align = row_alignment(static_cast<const float *>(a.y), a.y_pitch, a.y_bstride, a.batch);
+    const int col = c0 + R * lane;
+    const int hcol = c0 + kStrip + 4 * lane;
+    const bool has_halo = kHalo && 4 * lane < Q - 1;
+    const int i_end = r1 + P - 1;
+
+    float2 Z[SP][R];
+#pragma unroll
+    for (int m = 0; m < SP; ++m)
+#pragma unroll
+        for (int j = 0; j < R; ++j) Z[m][j] = make_float2(0.f, 0.f);
+    float nX[2][R], nH[2][4];
+#pragma unroll
+    for (int t = 0; t < 2; ++t)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) nH[t][j] = 0;
+    auto fetch = [&](int i) {
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+            const float *rowp = xb + static_cast<long long>(min(i + t, a.height - 1)) * a.x_pitch;
+#pragma unroll
+            for (int g = 0; g < R / 4; ++g) load_group<Tr>(rowp, col + 4 * g, a.width, x_vec, &nX[t][4 * g]);
+            if (has_halo) load_group<Tr>(rowp, hcol, a.width, x_vec, nH[t]);
+        }
+    };
+    fetch(r0);
+#pragma unroll 1
+    for (int i = r0; i < i_end; i += 2) {
+        float X[2][R], H[2][4];
+#pragma unroll
+        for (int t = 0; t < 2; ++t) {
+#pragma unroll
+            for (int j = 0; j < R; ++j) X[t][j] = nX[t][j];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) H[t][j] = nH[t][j];
+        }
+        if (i + 2 < i_end) fetch(i + 2);
+        // slot k holds output row (i+1)-k; pair m = slots (2m, 2m+1); all slots move up by two per iteration
+#pragma unroll
+        for (int q = 0; q < Q; ++q) {
+            float2 D0[R], D1[R];
+#pragma unroll
+            for (int j = 0; j < R; ++j) { D0[j] = make_float2(X[0][j], X[0][j]); D1[j] = make_float2(X[1][j], X[1][j]); }
+#pragma unroll
+            for (int m = SP - 1; m >= 0; --m) {
+                const float2 wa = taps.a[m * Q + q];      // row i+1 reaches slots 2m, 2m+1 through filter rows 2m, 2m+1
+                const float2 wb = taps.b[m * Q + q];      // row i   reaches them through filter rows 2m-1, 2m
+#pragma unroll
+                for (int j = 0; j < R; ++j) {
+                    float2 z = (q == 0) ? (m > 0 ? Z[m - 1][j] : make_float2(0.f, 0.f)) : Z[m][j];
+                    z = __ffma2_rn(D1[j], wa, z);
+                    Z[m][j] = __ffma2_rn(D0[j], wb, z);
+                }
+            }
+            if (q < Q - 1) {
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    const float send = (lane == 0) ? H[t][0] : X[t][0];
+                    const float in0 = __shfl_sync(kFullMask, send, (lane + 1) & (kLanes - 1));
+#pragma unroll
+                    for (int j = 0; j < R - 1; ++j) X[t][j] = X[t][j + 1];
+                    X[t][R - 1] = in0;
+                    float in1 = 0;
+                    if (kHaloChain) in1 = __shfl_down_sync(kFullMask, H[t][0], 1);
+                    H[t][0] = H[t][1]; H[t][1] = H[t][2]; H[t][2] = H[t][3]; H[t][3] = in1;
+                }
+            }
+        }
+        // slots P-1 (output row i-P+2) and P (output row i-P+1) are complete
+        float lo[R], hi[R];
+#pragma unroll
+        for (int j = 0; j < R; ++j) {
+            hi[j] = (P & 1) ? Z[(P - 1) / 2][j].x : Z[(P - 1) / 2][j].y;     // slot P-1
+            lo[j] = (P & 1) ? Z[P / 2][j].y : Z[P / 2][j].x;                 // slot P
+        }
+        const int rl = i - (P - 1), rh = rl + 1;
+#pragma unroll
+        for (int g = 0; g < R / 4; ++g) {
+            if (rl >= r0 && rl < r1) store_group<Tr>(yb + static_cast<long long>(rl) * a.y_pitch, col + 4 * g, a.out_w, y_align, &lo[4 * g]);
+            if (rh >= r0 && rh < r1) store_group<Tr>(yb + static_cast<long long>(rh) * a.y_pitch, col + 4 * g, a.out_w, y_align, &hi[4 * g]);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
 // IS / SBM
 // ---------------------------------------------------------------------------
 template <int Q, int R>
@@ -526,6 +652,25 @@ cudaError_t launch_conv2d_osis(const Conv2DArgs &a, const typename Tr::taps_t &t
     return cudaGetLastError();
 }
 
+template <int P, int Q>
+cudaError_t launch_conv2d_os_rowpair(const Conv2DArgs &a, const float *w, cudaStream_t s)
+{
+    constexpr int R = 4, MINB = 4;
+    TapsRowPairs t;
+    auto tap = [&](int p, int q) { return (p >= 0 && p < P) ? w[p * Q + q] : 0.f; };
+    for (int m = 0; m < 8; ++m)
+        for (int q = 0; q < Q; ++q) {
+            t.a[m * Q + q] = make_float2(tap(2 * m, q), tap(2 * m + 1, q));
+            t.b[m * Q + q] = make_float2(tap(2 * m - 1, q), tap(2 * m, q));
+        }
+    const int strips = (a.out_w + kLanes * R - 1) / (kLanes * R);
+    const int band_h = pick_band_height(a.out_h, static_cast<long long>(strips) * a.batch, P, Q);
+    dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + band_h - 1) / band_h, a.batch);
+    if (grid.y > 65535) return cudaErrorInvalidConfiguration;
+    conv2d_os_rowpair_kernel<P, Q, R, MINB><<<grid, kThreads2, 0, s>>>(a, t, band_h);
+    return cudaGetLastError();
+}
+
 template <typename Tr, int DESIGN, int P, int Q>
 cudaError_t launch_conv2d_pq(const Conv2DArgs &a, const typename Tr::taps_t &taps, cudaStream_t s)
 {
@@ -547,6 +692,8 @@ cudaError_t launch_conv2d_pq(const Conv2DArgs &a, const typename Tr::taps_t &tap
         return cudaGetLastError();
     }
     using Sh = Shape2D<Tr, DESIGN, P, Q>;
+    if constexpr (std::is_same<Tr, F32Traits>::value && DESIGN == SYSCONV_OS && P >= 9)
+        return launch_conv2d_os_rowpair<P, Q>(a, taps.w, s);
     if (Sh::kAlsoNarrow) {
         // small image: with eight PEs per lane there would be fewer than ~8 warps per SM even with the
         // shortest bands, so take four PEs per lane
