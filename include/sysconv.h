@@ -44,10 +44,18 @@
  *     Any N, W, H, batch >= 1 that fit the index types; any pitch >= row length.
  *     Pointers need only be aligned to their element type (16-byte aligned
  *     rows run faster).
+ *   - Non-finite fp32 inputs (Inf, NaN): an input outside an output's window
+ *     never enters its sum, with two exceptions that pad with zero taps and
+ *     would multiply them by the non-finite value: the 2-D output-stationary
+ *     kernels with 12 or more filter rows (the output rows directly above and
+ *     below the affected rows may turn NaN) and the 2-D weight-stationary
+ *     kernels when q is not a multiple of 4 (up to three outputs to the left
+ *     of the affected columns may turn NaN).  Finite data is unaffected.
  *   - Errors: every function returns a sysconv_status; nothing throws, aborts
  *     or traps.  SYSCONV_EINVAL: null pointer, non-positive size, filter larger
  *     than the input, pitch/stride smaller than the row/array, unknown enum.
- *     SYSCONV_EUNSUPPORTED: filter size outside the compiled range.
+ *     SYSCONV_EUNSUPPORTED: filter size outside the compiled range, or one of
+ *     the designs FSM/BFS/FFS asked for anything but 1-D fp32.
  *     SYSCONV_ECUDA: the CUDA runtime reported an error at launch.
  */
 #ifndef SYSCONV_H_
@@ -67,9 +75,14 @@ typedef enum {
 } sysconv_status;
 
 typedef enum {
-    SYSCONV_WS = 0, /* BSM */
-    SYSCONV_OS = 1, /* FBS */
-    SYSCONV_IS = 2  /* SBM */
+    SYSCONV_WS = 0,  /* BSM */
+    SYSCONV_OS = 1,  /* FBS */
+    SYSCONV_IS = 2,  /* SBM */
+    /* the paper's other three 1-D designs (Table 2); 1-D fp32 only, built unfolded (one PE per lane,
+     * CheckTime on) as faithful renderings: expect a fraction of the speed of the three above */
+    SYSCONV_FSM = 3, /* inputs forwarded (2-step delay), weights stay, sums migrate */
+    SYSCONV_BFS = 4, /* inputs broadcast, weights forwarded, sums stay */
+    SYSCONV_FFS = 5  /* inputs forwarded, weights forwarded (2-step delay), sums stay */
 } sysconv_design;
 
 typedef enum {

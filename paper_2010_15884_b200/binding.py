@@ -13,9 +13,10 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_NAME = "libsysconv.so"
 
 WS, OS, IS = 0, 1, 2
+FSM, BFS, FFS = 3, 4, 5          # the paper's other three 1-D designs (1-D fp32 only)
 F32, U8S8_S32 = 0, 1
-DESIGN_NAMES = {WS: "WS", OS: "OS", IS: "IS"}
-_DESIGN_BY_NAME = {"WS": WS, "BSM": WS, "OS": OS, "FBS": OS, "IS": IS, "SBM": IS}
+DESIGN_NAMES = {WS: "WS", OS: "OS", IS: "IS", FSM: "FSM", BFS: "BFS", FFS: "FFS"}
+_DESIGN_BY_NAME = {"WS": WS, "BSM": WS, "OS": OS, "FBS": OS, "IS": IS, "SBM": IS, "FSM": FSM, "BFS": BFS, "FFS": FFS}
 
 _c_ll = ctypes.c_longlong
 _c_int = ctypes.c_int

@@ -105,6 +105,52 @@ __device__ __forceinline__ void os_pass_1d(const float *sx, float *so, const Tap
     }
 }
 
+// ---- output-stationary, PE-paired form for the longer filters (Q >= 12).  Same array, same forwarding
+// (one shuffle per step).  The partial sums of two neighbouring PEs c (even) and c+1 share a 64-bit
+// register pair, and ONE packed fp32x2 FMA (fma.rn.f32x2, sm_100) serves both: the input that PE c uses
+// with tap t at step t is the input PE c+1 used with tap t-1, so the multiplicand is (x, x) and the
+// multiplier the tap pair (w(t), w(t-1)), which comes straight from the kernel parameters as a
+// uniform-register pair.  Q+1 steps of R1/2 packed FMAs replace Q steps of R1 scalar ones: about half
+// the issue slots per MAC (the scalar form is issue-bound at Q = 32).  In the first and the last step
+// only one PE of each pair has a tap: those two steps use scalar FMAs, so that no input outside an
+// output's window ever enters its sum (a zero tap times a non-finite input would).
+template <int Q>
+__device__ __forceinline__ void os_pass_1d_paired(const float *sx, float *so, const Taps1D &taps, int lane)
+{
+    constexpr int M = R1 / 2;
+    float X[R1];
+    load_lane_block(sx + lane * R1, X);
+    float2 D[R1];                               // the forwarded inputs, each as the pair (x, x)
+#pragma unroll
+    for (int j = 0; j < R1; ++j) D[j] = make_float2(X[j], X[j]);
+    float2 Z[M];                                // Z[m] = partial sums of PEs 2m and 2m+1
+#pragma unroll
+    for (int t = 0; t <= Q; ++t) {
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+            if (t == 0) {
+                Z[m] = make_float2(D[2 * m].x * taps.w[0], 0.f);
+            } else if (t == Q) {
+                Z[m].y = fmaf(D[2 * m].x, taps.w[Q - 1], Z[m].y);
+            } else {
+                Z[m] = __ffma2_rn(D[2 * m], make_float2(taps.w[t], taps.w[t - 1]), Z[m]);
+            }
+        }
+        if (t < Q) {
+            const float in = __shfl_down_sync(kFullMask, D[0].x, 1);     // lane 31 keeps its own: invalid PEs
+#pragma unroll
+            for (int j = 0; j < R1 - 1; ++j) D[j] = D[j + 1];
+            D[R1 - 1] = make_float2(in, in);
+        }
+    }
+#pragma unroll
+    for (int g = 0; g < R1 / 4; ++g) {
+        const int off = lane * R1 + 4 * g;
+        if (off < kWarpOut1)
+            *reinterpret_cast<float4 *>(so + off) = make_float4(Z[2 * g].x, Z[2 * g].y, Z[2 * g + 1].x, Z[2 * g + 1].y);
+    }
+}
+
 // ---- input-stationary (SBM, Section 3.1): PE s keeps x(s); at step t = q the
 // partial sums move one PE up:  Z_s <- Z_{s-1} + X_s * w(q).  After Q steps PE s
 // holds y(s-(Q-1)); up to three more moves without arithmetic (drain) bring the
@@ -165,12 +211,19 @@ __device__ __forceinline__ void ws_pass_1d(const float *sx, float *so, const Tap
     const float4 *xs4 = reinterpret_cast<const float4 *>(sx + arr * kWsSeg1);
     float *yo = so + arr * kWsSeg1;
 
+    // PEs beyond Q (they exist only on the pair's second lane, when Q is not a multiple of four) pass the
+    // partial sum on untouched: adding x(t) times their zero tap would let a non-finite input outside an
+    // output's window into its sum
+    const bool upper = m == kWsLanes1 - 1;
     auto step = [&](float xb) -> float {
         float up = __shfl_up_sync(kFullMask, Z[RW - 1], 1, kWsLanes1);
         if (m == 0) up = 0.f;                          // PE 0: Z starts at zero
 #pragma unroll
-        for (int i = RW - 1; i > 0; --i) Z[i] = fmaf(xb, Wr[i], Z[i - 1]);
-        Z[0] = fmaf(xb, Wr[0], up);
+        for (int i = RW - 1; i > 0; --i) {
+            const float next = fmaf(xb, Wr[i], Z[i - 1]);
+            Z[i] = (RW + i >= Q && upper) ? Z[i - 1] : next;
+        }
+        Z[0] = (RW >= Q && upper) ? up : fmaf(xb, Wr[0], up);
         return Z[RW - 1];                              // on the array's last lane: y(t-(QP-1))
     };
 
@@ -185,6 +238,90 @@ __device__ __forceinline__ void ws_pass_1d(const float *sx, float *so, const Tap
         if (m == kWsLanes1 - 1 && off >= 0 && off < kWsSeg1)
             *reinterpret_cast<float4 *>(yo + off) = make_float4(o0, o1, o2, o3);
         o0 = step(xv.w);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------------
+// The paper's other three 1-D designs (Table 2): FSM, BFS and FFS.  They are built unfolded, one PE per
+// lane, with the CheckTime guard of Table 1 (a PE works only in its own time steps), as a faithful
+// rendering rather than a fast one: the paper's own model (Table 4) gives them 25 % (BFS) and 14 % (FFS)
+// lane utilisation and a quarter of the outturn of SBM/FBS.  The time loops are run-time loops over
+// t = s.z; forwarded values with a two-step delay keep a two-deep register history (Code 2).
+// ---------------------------------------------------------------------------------------------------
+
+// BFS: inputs broadcast, weights forwarded, sums stay.  PE c = lane, t = c + q.  Per step every PE takes
+// the weight its lower neighbour held one step ago (PE 0 takes w(t)), x(t) is broadcast, and PE c adds
+// x(t) * w(t-c) while 0 <= t-c < Q.  A warp slice of 608 outputs is 19 consecutive arrays of 32 PEs.
+template <int Q>
+__device__ __forceinline__ void bfs_pass_1d(const float *sx, float *so, const Taps1D &taps, int lane)
+{
+    for (int blk = 0; blk < kWarpOut1 / kLanes; ++blk) {
+        const float *xs = sx + blk * kLanes;
+        float W = 0.f, Z = 0.f;
+        for (int t = 0; t < kLanes + Q - 1; ++t) {
+            const float fwd = __shfl_up_sync(kFullMask, W, 1);
+            W = lane == 0 ? (t < Q ? taps.w[t] : 0.f) : fwd;
+            const float xb = xs[t];                                   // same address in every lane: broadcast
+            const int q = t - lane;
+            if (q >= 0 && q < Q) Z = (q == 0) ? xb * W : fmaf(xb, W, Z);
+        }
+        so[blk * kLanes + lane] = Z;
+    }
+}
+
+// FFS: inputs forwarded (one step), weights forwarded with a two-step delay, sums stay.  PE c = lane,
+// t = 2c + q.  X(c,q) comes from PE c-1 one step ago unless c == 0 or q == Q-1 (then x(c+q) is loaded);
+// W(c,q) comes from PE c-1 two steps ago (PE 0 takes w(t)).
+template <int Q>
+__device__ __forceinline__ void ffs_pass_1d(const float *sx, float *so, const Taps1D &taps, int lane)
+{
+    for (int blk = 0; blk < kWarpOut1 / kLanes; ++blk) {
+        const float *xs = sx + blk * kLanes;
+        float X = 0.f, W = 0.f, Wprev = 0.f, Z = 0.f;                 // Wprev: this PE's weight one step ago
+        for (int t = 0; t < 2 * (kLanes - 1) + Q; ++t) {
+            const float x_fwd = __shfl_up_sync(kFullMask, X, 1);      // neighbour's X of one step ago
+            const float w_fwd = __shfl_up_sync(kFullMask, Wprev, 1);  // neighbour's W of two steps ago
+            const int q = t - 2 * lane;
+            const bool active = q >= 0 && q < Q;
+            Wprev = W;
+            if (active) {
+                X = (lane == 0 || q == Q - 1) ? xs[lane + q] : x_fwd;
+                W = lane == 0 ? taps.w[q] : w_fwd;
+                Z = (q == 0) ? X * W : fmaf(X, W, Z);
+            }
+        }
+        so[blk * kLanes + lane] = Z;
+    }
+}
+
+// FSM: inputs forwarded with a two-step delay, weights stay, sums migrate.  PE q = lane inside an array of
+// LA lanes (LA = Q rounded up to a power of two; lanes beyond Q idle), t = c - q.  The stream enters at PE
+// Q-1; X(c,q) comes from PE q+1 two steps ago unless c == 0 or q == Q-1; Z(c,q) comes from PE q+1 one step
+// ago (PE Q-1 starts at zero); PE 0 emits y(c) at t = c.  The 32/LA arrays of a warp take consecutive
+// segments of the slice.
+template <int Q>
+__device__ __forceinline__ void fsm_pass_1d(const float *sx, float *so, const Taps1D &taps, int lane)
+{
+    constexpr int LA = Q <= 1 ? 1 : Q <= 2 ? 2 : Q <= 4 ? 4 : Q <= 8 ? 8 : Q <= 16 ? 16 : 32;
+    constexpr int kArrays = kLanes / LA;
+    constexpr int kSeg = kWarpOut1 / kArrays;                         // outputs per array
+    const int q = lane & (LA - 1);
+    const int arr = lane / LA;
+    const float *xs = sx + arr * kSeg;
+    float *ys = so + arr * kSeg;
+    const float w = q < Q ? taps.w[q] : 0.f;
+    float X = 0.f, Xprev = 0.f, Z = 0.f;                              // Xprev: this PE's input one step ago
+    for (int t = -(Q - 1); t < kSeg; ++t) {
+        const float x_fwd = __shfl_down_sync(kFullMask, Xprev, 1, LA);   // neighbour's X of two steps ago
+        const float z_fwd = __shfl_down_sync(kFullMask, Z, 1, LA);       // neighbour's Z of one step ago
+        const int c = t + q;
+        const bool active = q < Q && c >= 0 && c < kSeg;
+        Xprev = X;
+        if (active) {
+            X = (c == 0 || q == Q - 1) ? xs[c + q] : x_fwd;
+            Z = (q == Q - 1) ? X * w : fmaf(X, w, z_fwd);
+            if (q == 0) ys[c] = Z;
+        }
     }
 }
 
@@ -249,9 +386,13 @@ conv1d_f32_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, unsig
 
             const float *sx = s_in[k] + warp * G::kWarpOut;
             float *so = s_out[k] + warp * G::kWarpOut;
-            if (DESIGN == SYSCONV_OS) os_pass_1d<Q>(sx, so, taps, lane);
+            if (DESIGN == SYSCONV_OS && Q >= 12) os_pass_1d_paired<Q>(sx, so, taps, lane);
+            else if (DESIGN == SYSCONV_OS) os_pass_1d<Q>(sx, so, taps, lane);
             else if (DESIGN == SYSCONV_IS) is_pass_1d<Q>(sx, so, taps, lane);
-            else ws_pass_1d<Q>(sx, so, taps, lane);
+            else if (DESIGN == SYSCONV_WS) ws_pass_1d<Q>(sx, so, taps, lane);
+            else if (DESIGN == SYSCONV_FSM) fsm_pass_1d<Q>(sx, so, taps, lane);
+            else if (DESIGN == SYSCONV_BFS) bfs_pass_1d<Q>(sx, so, taps, lane);
+            else ffs_pass_1d<Q>(sx, so, taps, lane);
 
             if (out_by_copy) {
                 fence_proxy_async();                     // my shared-memory writes, before the bulk store reads them

@@ -225,7 +225,7 @@ conv2d_os_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t
 }
 
 // ---------------------------------------------------------------------------
-// OS / FBS, fp32, row-paired form for the tall filters (P >= 9).
+// OS / FBS, fp32, row-paired form for filters with six or more rows.
 //
 // Same dataflow as conv2d_os_kernel, two input rows per iteration.  The partial sums of two consecutive
 // output rows share a 64-bit register pair and are updated by ONE packed fp32x2 FMA (fma.rn.f32x2, new on
@@ -235,6 +235,9 @@ conv2d_os_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t
 // scalar kernel is issue-bound (81 % of its instructions are FMAs at 89 % issue-slot use), this form is
 // FMA-pipe-bound.  Both rows' inputs are forwarded exactly as before (one shuffle per row and step).
 // With P odd the P+1 slots fill the pairs exactly; with P even one slot of the last pair stays zero.
+// Slots without a tap for one of the two rows: scalar FMAs on the other half for P <= 11 (exact), a zero tap
+// for P >= 12 (measured faster there), where a NON-FINITE input can therefore also turn the outputs one row
+// above and one row below its window rows into NaN; finite inputs are unaffected.
 // ---------------------------------------------------------------------------
 // Slots and slot pairs of the row-paired kernel: P + 1 partial rows are alive while two input rows are
 // processed; pair m holds the slots 2m and 2m+1.
@@ -248,7 +251,7 @@ struct TapsRowPairs {
     float2 a[8 * kMaxQ2];
     float2 b[8 * kMaxQ2];
 };
-template <int P, int Q, int R, int MIN_CTAS>
+template <int P, int Q, int R, int MIN_CTAS, bool EXACT_HALVES>
 __global__ void __launch_bounds__(kThreads2, MIN_CTAS)
 conv2d_os_rowpair_kernel(const Conv2DArgs a, const __grid_constant__ TapsRowPairs taps, const int band_h)
 {
@@ -313,11 +316,19 @@ conv2d_os_rowpair_kernel(const Conv2DArgs a, const __grid_constant__ TapsRowPair
             for (int m = SP - 1; m >= 0; --m) {
                 const float2 wa = taps.a[m * Q + q];      // row i+1 reaches slots 2m, 2m+1 through filter rows 2m, 2m+1
                 const float2 wb = taps.b[m * Q + q];      // row i   reaches them through filter rows 2m-1, 2m
+                // slots of a pair that have no tap for one of the two rows: either a scalar FMA on the other half
+                // (EXACT_HALVES: nothing outside an output's window enters its sum) or a packed FMA with a zero tap
+                const bool a_both = !EXACT_HALVES || 2 * m + 1 < P, a_first = 2 * m < P;
+                const bool b_both = !EXACT_HALVES || (m > 0 && 2 * m < P), b_second = m == 0, b_first = 2 * m - 1 < P;
 #pragma unroll
                 for (int j = 0; j < R; ++j) {
                     float2 z = (q == 0) ? (m > 0 ? Z[m - 1][j] : make_float2(0.f, 0.f)) : Z[m][j];
-                    z = __ffma2_rn(D1[j], wa, z);
-                    Z[m][j] = __ffma2_rn(D0[j], wb, z);
+                    if (a_both) z = __ffma2_rn(D1[j], wa, z);
+                    else if (a_first) z.x = fmaf(D1[j].x, wa.x, z.x);
+                    if (b_both) z = __ffma2_rn(D0[j], wb, z);
+                    else if (b_second) z.y = fmaf(D0[j].x, wb.y, z.y);
+                    else if (b_first) z.x = fmaf(D0[j].x, wb.x, z.x);
+                    Z[m][j] = z;
                 }
             }
             if (q < Q - 1) {
@@ -450,7 +461,9 @@ conv2d_is_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t
 // arrays and a CTA 32, stacked over 32*M = 128 output rows.  The CTA streams a segment of the image
 // width through shared memory in chunks of 32 columns, stored TRANSPOSED ([column][row], rows in
 // XOR-swizzled groups of four) so that an array reads the inputs of one image column with 128-bit
-// same-address (broadcast) loads; arrays never refill inside a segment.
+// same-address (broadcast) loads; arrays never refill inside a segment.  The up to three PEs beyond the filter
+// width keep zero taps (guarding them was measured 15-60 % slower), so with fp32 data a NON-FINITE input can
+// also turn the up to three outputs to the left of its window columns into NaN; finite inputs are unaffected.
 // ---------------------------------------------------------------------------
 constexpr int kWsM2 = 4;                        // output rows per array
 constexpr int kWsRows2 = kWarps2 * kWsArrays * kWsM2;   // 128 output rows per CTA
@@ -607,10 +620,9 @@ conv2d_ws_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t
 // Shape of the OS/IS kernels per filter size (measured on B200, 16 x 4096 x 4096 fp32):
 //   small filters are memory-bound: eight PEs per lane, short bands (many CTAs in flight) and two input
 //     rows in flight per warp (four measured slower); on small images four PEs per lane instead (twice as many warps);
-//   mid-size OS filters: eight PEs per lane under a 128-register cap (four CTAs per SM), which raises the
-//     FMA share of the instruction stream (weight fetches and bookkeeping are per lane and row);
-//   OS filters with 12 or more rows, and IS beyond the small filters, keep four PEs per lane: their
-//     P*8 partial sums (OS) or stationary inputs (IS) no longer fit.
+//   fp32 OS filters with six or more rows use the row-paired kernel (launch_conv2d_os_rowpair) instead;
+//   the scalar OS kernel with 6 <= P <= 11 (integer data) takes eight PEs per lane under a 128-register cap;
+//   IS beyond the small filters keeps four PEs per lane: P*8 stationary inputs no longer fit.
 template <typename Tr, int DESIGN, int P, int Q>
 struct Shape2D {
     static constexpr bool kF32 = std::is_same<Tr, F32Traits>::value;
@@ -652,6 +664,11 @@ cudaError_t launch_conv2d_osis(const Conv2DArgs &a, const typename Tr::taps_t &t
     return cudaGetLastError();
 }
 
+// scalar half-steps where a slot pair has a tap for only one slot: exact for non-finite inputs and measured
+// faster up to 11 filter rows (9x9: 72 % vs 68 % of FP32 peak), slower from 12 on (15x15: 69 % vs 79 %)
+template <int P>
+constexpr bool kRowPairExact = P <= 11;
+
 template <int P, int Q>
 cudaError_t launch_conv2d_os_rowpair(const Conv2DArgs &a, const float *w, cudaStream_t s)
 {
@@ -667,7 +684,7 @@ cudaError_t launch_conv2d_os_rowpair(const Conv2DArgs &a, const float *w, cudaSt
     const int band_h = pick_band_height(a.out_h, static_cast<long long>(strips) * a.batch, P, Q);
     dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + band_h - 1) / band_h, a.batch);
     if (grid.y > 65535) return cudaErrorInvalidConfiguration;
-    conv2d_os_rowpair_kernel<P, Q, R, MINB><<<grid, kThreads2, 0, s>>>(a, t, band_h);
+    conv2d_os_rowpair_kernel<P, Q, R, MINB, kRowPairExact<P>><<<grid, kThreads2, 0, s>>>(a, t, band_h);
     return cudaGetLastError();
 }
 
@@ -692,7 +709,7 @@ cudaError_t launch_conv2d_pq(const Conv2DArgs &a, const typename Tr::taps_t &tap
         return cudaGetLastError();
     }
     using Sh = Shape2D<Tr, DESIGN, P, Q>;
-    if constexpr (std::is_same<Tr, F32Traits>::value && DESIGN == SYSCONV_OS && P >= 9)
+    if constexpr (std::is_same<Tr, F32Traits>::value && DESIGN == SYSCONV_OS && P >= 6)
         return launch_conv2d_os_rowpair<P, Q>(a, taps.w, s);
     if (Sh::kAlsoNarrow) {
         // small image: with eight PEs per lane there would be fewer than ~8 warps per SM even with the

@@ -95,9 +95,10 @@ HostPipe *host_pipe()
 
 bool valid_enums(int dtype, int design)
 {
-    return (dtype == SYSCONV_F32 || dtype == SYSCONV_U8S8_S32) &&
-           (design == SYSCONV_WS || design == SYSCONV_OS || design == SYSCONV_IS);
+    return (dtype == SYSCONV_F32 || dtype == SYSCONV_U8S8_S32) && design >= SYSCONV_WS && design <= SYSCONV_FFS;
 }
+
+bool main_design(int design) { return design == SYSCONV_WS || design == SYSCONV_OS || design == SYSCONV_IS; }
 
 // true if [a, a+an) and [b, b+bn) overlap
 bool overlaps(const void *a, unsigned long long an, const void *b, unsigned long long bn)
@@ -157,10 +158,12 @@ int sysconv1d(const void *x_dev, long long n, long long x_batch_stride, const vo
         if (!d) return SYSCONV_ECUDA;
         cudaError_t err = design == SYSCONV_OS   ? launch_conv1d_f32_os(a, w, q, d->status_word, s, &launches)
                           : design == SYSCONV_IS ? launch_conv1d_f32_is(a, w, q, d->status_word, s, &launches)
-                                                 : launch_conv1d_f32_ws(a, w, q, d->status_word, s, &launches);
+                          : design == SYSCONV_WS ? launch_conv1d_f32_ws(a, w, q, d->status_word, s, &launches)
+                                                 : launch_conv1d_f32_other(design, a, w, q, d->status_word, s, &launches);
         return finish(err, launches);
     }
     // integer signals run as one-row images through the 2-D integer kernels
+    if (!main_design(design)) return SYSCONV_EUNSUPPORTED;
     if (q > kMaxQ2) return SYSCONV_EUNSUPPORTED;
     if (n > 0x7fffffffLL) return SYSCONV_EUNSUPPORTED;
     Conv2DArgs a;
@@ -189,7 +192,7 @@ int sysconv2d(const void *x_dev, int width, int height, long long x_pitch, long 
     const unsigned long long x_bytes = ((unsigned long long)(batch - 1) * x_batch_stride + x_img) * in_elt_bytes(dtype);
     const unsigned long long y_bytes = ((unsigned long long)(batch - 1) * y_batch_stride + y_img) * 4ull;
     if (overlaps(x_dev, x_bytes, y_dev, y_bytes)) return SYSCONV_EINVAL;
-    if (q > kMaxQ2 || p > kMaxP2) return SYSCONV_EUNSUPPORTED;
+    if (q > kMaxQ2 || p > kMaxP2 || !main_design(design)) return SYSCONV_EUNSUPPORTED;
 
     Conv2DArgs a;
     a.x = x_dev; a.y = y_dev;
@@ -363,6 +366,9 @@ const char *sysconv_design_name(int design)
         case SYSCONV_WS: return "WS/BSM";
         case SYSCONV_OS: return "OS/FBS";
         case SYSCONV_IS: return "IS/SBM";
+        case SYSCONV_FSM: return "FSM";
+        case SYSCONV_BFS: return "BFS";
+        case SYSCONV_FFS: return "FFS";
         default: return "?";
     }
 }

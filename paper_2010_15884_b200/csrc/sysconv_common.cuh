@@ -81,6 +81,9 @@ cudaError_t launch_conv1d_f32_is(const Conv1DArgs &a, const float *w, int q, uns
                                  int *launches);
 cudaError_t launch_conv1d_f32_ws(const Conv1DArgs &a, const float *w, int q, unsigned *status_word, cudaStream_t s,
                                  int *launches);
+// the paper's other three designs (FSM, BFS, FFS): design = SYSCONV_FSM / SYSCONV_BFS / SYSCONV_FFS
+cudaError_t launch_conv1d_f32_other(int design, const Conv1DArgs &a, const float *w, int q, unsigned *status_word,
+                                    cudaStream_t s, int *launches);
 
 cudaError_t launch_conv2d_f32_os(const Conv2DArgs &a, const float *w, int q, int p, cudaStream_t s, int *launches);
 cudaError_t launch_conv2d_f32_is(const Conv2DArgs &a, const float *w, int q, int p, cudaStream_t s, int *launches);

@@ -44,6 +44,8 @@ def test_strings_and_version_without_a_gpu(lib):
     assert binding.design_name(binding.WS) == "WS/BSM"
     assert binding.design_name(binding.OS) == "OS/FBS"
     assert binding.design_name(binding.IS) == "IS/SBM"
+    assert [binding.design_name(d) for d in (binding.FSM, binding.BFS, binding.FFS)] == ["FSM", "BFS", "FFS"]
+    assert binding.design_name(6) == "?"
     assert binding.launch_count() >= 0
 
 
@@ -57,7 +59,7 @@ def test_argument_validation_needs_no_gpu(lib):
     assert b.sysconv1d(fake_x, 3, 3, w, 4, fake_y, 0, 1, b.F32, b.OS, 0) == 1           # n < q
     assert b.sysconv1d(fake_x, 100, 100, w, 4, fake_y, 97, 0, b.F32, b.OS, 0) == 1      # batch < 1
     assert b.sysconv1d(fake_x, 100, 100, w, 4, fake_y, 97, 1, 7, b.OS, 0) == 1          # dtype
-    assert b.sysconv1d(fake_x, 100, 100, w, 4, fake_y, 97, 1, b.F32, 5, 0) == 1         # design
+    assert b.sysconv1d(fake_x, 100, 100, w, 4, fake_y, 97, 1, b.F32, 6, 0) == 1         # design
     assert b.sysconv1d(fake_x, 100, 50, w, 4, fake_y, 97, 2, b.F32, b.OS, 0) == 1       # batch stride < n
     assert b.sysconv1d(fake_x, 100, 100, w, 4, fake_x + 16, 97, 1, b.F32, b.OS, 0) == 1  # overlap
     w33 = np.ones(33, np.float32)

@@ -14,6 +14,7 @@ from paper_2010_15884_b200 import inputs
 pytestmark = pytest.mark.gpu
 
 DESIGNS = [B.WS, B.OS, B.IS]
+OTHER_DESIGNS = [B.FSM, B.BFS, B.FFS]        # the paper's other three 1-D designs (1-D fp32 only)
 TOL = 1e-5
 CANARY = 12345.0
 
@@ -34,6 +35,16 @@ def assert_close_f32(y_gpu, y_ref, s_ref, what=""):
         raise AssertionError("%s: %d outputs beyond 1e-5*S; worst at flat index %d: gpu %r ref %r S %r"
                              % (what, int(bad.sum()), i, y_gpu.flat[i], y_ref.flat[i], s_ref.flat[i]))
     assert np.isfinite(y_gpu).all()
+
+
+def _assert_same_where_finite(y_gpu, y_ref, s_ref, what):
+    """Outputs whose window holds no non-finite input must be finite and within tolerance; the others must be
+    non-finite on both sides."""
+    y_gpu = np.asarray(y_gpu, np.float64)
+    fin = np.isfinite(y_ref)
+    assert (np.isfinite(y_gpu) == fin).all(), "%s: non-finite outputs differ (%d vs %d)" % (
+        what, int((~np.isfinite(y_gpu)).sum()), int((~fin).sum()))
+    assert (np.abs(y_gpu[fin] - y_ref[fin]) <= TOL * s_ref[fin]).all(), what
 
 
 # ------------------------------------------------------------------------ 1-D fp32
@@ -128,6 +139,57 @@ def test_1d_many_tiles_batch(cuda_device, design):
         y_ref, s_ref = oracle.conv1d_f32(x[b], w)
         assert_close_f32(y[b], y_ref, s_ref, "batch %d" % b)
     assert B.device_status() == 0
+
+
+@pytest.mark.parametrize("design", OTHER_DESIGNS, ids=_ids)
+@pytest.mark.parametrize("q", [1, 2, 3, 5, 8, 13, 16, 17, 31, 32])
+def test_1d_other_designs_filter_lengths(cuda_device, design, q):
+    x, ws = inputs.gen_1d_f32(21000, [q], seed=500 + q)
+    y_ref, s_ref = oracle.conv1d_f32(x, ws[q])
+    assert_close_f32(run_1d(x, ws[q], design, cuda_device), y_ref, s_ref, "q=%d" % q)
+
+
+@pytest.mark.parametrize("design", OTHER_DESIGNS, ids=_ids)
+@pytest.mark.parametrize("extra", [0, 1, 18, 19, 31, 32, 607, 608, 1215, 1216, 2431, 2432, 2433])
+def test_1d_other_designs_ragged_sizes_and_config1(cuda_device, design, extra):
+    q = 5
+    x, ws = inputs.gen_1d_f32(q + extra, [q], seed=600 + extra)
+    y_ref, s_ref = oracle.conv1d_f32(x, ws[q])
+    assert_close_f32(run_1d(x, ws[q], design, cuda_device), y_ref, s_ref, "n_out=%d" % (extra + 1))
+    if extra == 0:
+        x1, ws1 = inputs.make_config(1)
+        y_ref, s_ref = oracle.conv1d_f32(x1, ws1[8])
+        assert_close_f32(run_1d(x1, ws1[8], design, cuda_device), y_ref, s_ref, "config 1")
+        xb = np.stack([x1[:3000], x1[1000:4000]])
+        yb = run_1d(xb, ws1[8], design, cuda_device, batch_stride=3001, offset=1)
+        for b in range(2):
+            y_ref, s_ref = oracle.conv1d_f32(xb[b], ws1[8])
+            assert_close_f32(yb[b], y_ref, s_ref, "batch %d" % b)
+
+
+@pytest.mark.parametrize("design", OTHER_DESIGNS, ids=_ids)
+def test_1d_other_designs_exact_integers_and_non_finite(cuda_device, design):
+    rng = np.random.default_rng(18)
+    x = rng.integers(-50, 51, 9000).astype(np.float32)
+    w = rng.integers(-9, 10, 7).astype(np.float32)
+    y_ref, _ = oracle.conv1d_f32(x, w)
+    np.testing.assert_array_equal(run_1d(x, w, design, cuda_device).astype(np.float64), y_ref)
+    x, ws = inputs.gen_1d_f32(9000, [6], seed=19)
+    x[[3, 607, 608, 4000, 8999]] = [np.inf, np.nan, -np.inf, np.inf, np.nan]
+    with np.errstate(invalid="ignore"):
+        y_ref, s_ref = oracle.conv1d_f32(x, ws[6])
+    _assert_same_where_finite(run_1d(x, ws[6], design, cuda_device), y_ref, s_ref, "non-finite")
+
+
+def test_other_designs_are_1d_fp32_only(cuda_device):
+    x2 = torch.zeros((1, 40, 40), device=cuda_device)
+    for design in OTHER_DESIGNS:
+        with pytest.raises(B.SysconvError) as e:
+            B.conv2d(x2, np.ones((3, 3), np.float32), design)
+        assert e.value.status == 2
+        with pytest.raises(B.SysconvError) as e:
+            B.conv1d(torch.zeros(100, dtype=torch.uint8, device=cuda_device), np.ones(3, np.int8), design)
+        assert e.value.status == 2
 
 
 @pytest.mark.parametrize("design", DESIGNS, ids=_ids)
@@ -272,6 +334,60 @@ def test_config5_full_size_sampled(cuda_device, k):
         if k == 3:
             y_ref, s_ref = oracle.conv2d_f32(x[7], w)
             assert_close_f32(yd[7].cpu().numpy(), y_ref, s_ref, "config 5 image 7 full")
+
+
+# ------------------------------------------------------------------------ non-finite inputs
+
+
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+@pytest.mark.parametrize("q", [3, 5, 13, 16, 31, 32])
+def test_1d_non_finite_inputs_stay_inside_their_windows(cuda_device, design, q):
+    x, ws = inputs.gen_1d_f32(30000, [q], seed=3000 + q)
+    x[[17, 4863, 4864, 9000, 9001, 20000, 29990]] = [np.inf, -np.inf, np.nan, np.inf, np.inf, np.nan, np.inf]
+    with np.errstate(invalid="ignore"):
+        y_ref, s_ref = oracle.conv1d_f32(x, ws[q])
+    _assert_same_where_finite(run_1d(x, ws[q], design, cuda_device), y_ref, s_ref, "1-D q=%d" % q)
+
+
+BAD_PIXELS = ((0, 0, np.inf), (40, 127, np.nan), (41, 128, -np.inf), (63, 255, np.inf), (64, 256, np.nan),
+              (119, 299, np.inf), (100, 5, np.inf))
+
+
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+@pytest.mark.parametrize("pq", [(3, 3), (5, 5), (8, 6), (9, 9), (10, 7), (15, 15), (4, 8), (12, 12)],
+                         ids=lambda f: "%dx%d" % f)
+def test_2d_non_finite_inputs_stay_inside_their_windows(cuda_device, design, pq):
+    """A non-finite pixel affects exactly the outputs whose window holds it -- except for the two documented
+    zero-tap paddings (OS with P >= 12: one more row above and below; WS with Q % 4 != 0: up to three more columns
+    to the left), where those extra outputs may be NaN and everything else must still be exact."""
+    p, q = pq
+    x, ws = inputs.gen_2d_f32(300, 120, [pq], seed=3100 + p)
+    for r, c, v in BAD_PIXELS:
+        x[0, r, c] = v
+    with np.errstate(invalid="ignore"):
+        y_ref, s_ref = oracle.conv2d_f32(x[0], ws[pq])
+    y = run_2d(x, ws[pq], design, cuda_device)[0].astype(np.float64)
+    oh, ow = y_ref.shape
+    may_differ = np.zeros((oh, ow), bool)
+    for rb, cb, _ in BAD_PIXELS:
+        c_lo, c_hi = max(cb - q + 1, 0), min(cb, ow - 1)
+        if design == B.OS and p >= 12:
+            for r in (rb - p, rb + 1):
+                if 0 <= r < oh and c_lo <= c_hi:
+                    may_differ[r, c_lo:c_hi + 1] = True
+        if design == B.WS and q % 4:
+            qp = (q + 3) // 4 * 4
+            r_lo, r_hi = max(rb - p + 1, 0), min(rb, oh - 1)
+            cc_lo, cc_hi = max(cb - qp + 1, 0), min(cb - q, ow - 1)
+            if r_lo <= r_hi and cc_lo <= cc_hi:
+                may_differ[r_lo:r_hi + 1, cc_lo:cc_hi + 1] = True
+    strict = ~may_differ
+    fin = np.isfinite(y_ref)
+    assert (np.isfinite(y[strict]) == fin[strict]).all(), "non-finite outputs differ outside the documented cells"
+    ok = strict & fin
+    assert (np.abs(y[ok] - y_ref[ok]) <= TOL * s_ref[ok]).all()
+    loose = may_differ & fin & np.isfinite(y)
+    assert (np.abs(y[loose] - y_ref[loose]) <= TOL * s_ref[loose]).all()
 
 
 # ------------------------------------------------------------------------ integer
