@@ -410,6 +410,7 @@ def run_ours(args):
             torch.cuda.empty_cache()
             line["detail"] = all_config_detail(device, hbm_gbs, peak_kind, sm_max, skip=cfg_id,
                                                reps=args.detail_reps)
+            line["six_designs_n2p24"] = six_designs_table(device, args.detail_reps)
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -485,6 +486,44 @@ def run_e2e(cfg_id, device, args, world):
             "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": steps,
             "ms_per_step": round(ms / steps, 3),
             "path": "sysconv1d_host/sysconv2d_host: pinned host -> device workspace -> kernel -> pinned host"}
+
+
+def six_designs_table(device, reps):
+    """The shape of the paper's Table 3 / Table 4 experiment on B200: the six 1-D designs at filter sizes 2 and 5,
+    throughput relative to FBS (the paper compared with the GEN9.5 sampler, which does not exist here), beside the
+    analytical model's outturn and lane utilisation for 16 outputs, filter size 5 (Table 4)."""
+    import torch
+    from paper_2010_15884_b200 import binding as B
+    from paper_2010_15884_b200 import inputs
+    model = {"SBM": (3.2, 80), "BSM": (0.8, 80), "FSM": (0.8, 80), "BFS": (0.8, 25), "FFS": (0.46, 14), "FBS": (3.2, 100)}
+    enum = {"SBM": B.IS, "BSM": B.WS, "FSM": B.FSM, "BFS": B.BFS, "FFS": B.FFS, "FBS": B.OS}
+    n = 1 << 24
+    x, ws = inputs.gen_1d_f32(n, [2, 5], seed=5)
+    xd = torch.from_numpy(x).to(device)
+    stream = torch.cuda.current_stream().cuda_stream
+    rows = []
+    for q, w in ws.items():
+        yd = torch.empty(n - q + 1, dtype=torch.float32, device=device)
+        times = {}
+        for name, d in enum.items():
+            def launch(d=d, w=w, q=q, yd=yd):
+                st = B.sysconv1d(xd.data_ptr(), n, n, w, q, yd.data_ptr(), n - q + 1, 1, B.F32, d, stream)
+                if st != 0:
+                    raise B.SysconvError(st, "sysconv1d")
+            for _ in range(3):
+                launch()
+            ts = []
+            for _ in range(reps):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); launch(); e1.record(); e1.synchronize()
+                ts.append(e0.elapsed_time(e1))
+            times[name] = statistics.median(ts)
+        for name in enum:
+            rows.append({"design": name, "filter": q, "ms": round(times[name], 5),
+                         "gpix_s": round((n - q + 1) / (times[name] * 1e-3) / 1e9, 2),
+                         "relative_to_FBS": round(times["FBS"] / times[name], 3),
+                         "model_outturn_q5": model[name][0], "model_utilisation_pct_q5": model[name][1]})
+    return rows
 
 
 def all_config_detail(device, hbm_gbs, peak_kind, sm_max, skip, reps):

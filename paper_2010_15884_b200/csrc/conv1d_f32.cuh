@@ -38,12 +38,12 @@ struct Geo1D {
     static constexpr int kTileOut = kWarps * kWarpOut;     // outputs per CTA tile
     static constexpr int kTileIn = kTileOut + kHalo1;      // inputs per CTA tile
 };
-// shape used by the library (measured best on B200): OS/IS two warps and two tiles per CTA,
-// WS one warp and one (twice as large) tile per CTA
-template <int DESIGN>
+// shape used by the library (measured best on B200): two warps and two tiles per CTA; WS one warp per CTA
+// with one (twice as large) tile, two for the longer filters
+template <int DESIGN, int Q>
 struct DefaultShape1D {
     static constexpr int kWarps = DESIGN == SYSCONV_WS ? 1 : 2;
-    static constexpr int kTiles = DESIGN == SYSCONV_WS ? 1 : 2;
+    static constexpr int kTiles = DESIGN == SYSCONV_WS ? (Q > 16 ? 2 : 1) : 2;
 };
 
 // ---- ordinary-load staging (ragged or unaligned tiles) ------------------------
@@ -193,12 +193,21 @@ __device__ __forceinline__ void is_pass_1d(const float *sx, float *so, const Tap
 // array length QP = 2*RW is kept a multiple of four so that outputs leave as
 // aligned 128-bit words); array a streams the 76-output segment a of the warp's
 // 1216-output slice.  The broadcast is a same-address shared-memory read.
+//
+// Arrays neither fill nor drain separately: every array runs exactly the 76 steps
+// of its segment.  What array a+1 emits during its first QP-1 steps (sums over its
+// own inputs only) are the missing parts of the QP-1 sums still in flight in array a
+// when it stops, so they are stored into segment a's tail and array a adds its
+// registers to them afterwards.  Only the last array of the slice has no successor:
+// its tail gets the missing taps from a short direct sum over the slice's halo.
 template <int Q>
 __device__ __forceinline__ void ws_pass_1d(const float *sx, float *so, const Taps1D &taps, int lane)
 {
     constexpr int RW = 2 * ((Q + 3) / 4);
     constexpr int QP = RW * kWsLanes1;
-    constexpr int kGroups = (kWsSeg1 + QP) / 4;       // time steps in groups of four
+    constexpr int kGroups = kWsSeg1 / 4;              // 76 time steps in groups of four
+    constexpr int kSlice = kWsArrays1 * kWsSeg1;      // 1216 outputs
+    static_assert(QP <= kHalo1 && QP <= kWsSeg1, "array longer than the halo or the segment");
     const int m = lane & (kWsLanes1 - 1);
     const int arr = lane / kWsLanes1;
     float Wr[RW], Z[RW];
@@ -234,10 +243,30 @@ __device__ __forceinline__ void ws_pass_1d(const float *sx, float *so, const Tap
         const float o1 = step(xv.x);
         const float o2 = step(xv.y);
         const float o3 = step(xv.z);
-        const int off = 4 * k - QP;                    // outputs 4k-QP .. 4k-QP+3 are now complete
-        if (m == kWsLanes1 - 1 && off >= 0 && off < kWsSeg1)
+        // outputs 4k-QP .. 4k-QP+3 of this segment; negative positions are the tail of the previous
+        // segment and receive this array's share of those sums (the first array of the slice has no
+        // predecessor in the slice: the previous slice patches its own tail)
+        const int off = 4 * k - QP;
+        if (upper && (off >= 0 || arr > 0))
             *reinterpret_cast<float4 *>(yo + off) = make_float4(o0, o1, o2, o3);
         o0 = step(xv.w);
+    }
+    // The last array's tail has no successor: store the taps it is missing, summed directly over the halo
+    // (output c = kSlice-1-j lacks the taps k > j); position kSlice-QP lacks nothing.
+    if (lane < QP) {
+        const int c = kSlice - 1 - lane;
+        float acc = 0.f;
+#pragma unroll
+        for (int k = 1; k < Q; ++k)
+            if (k > lane) acc = fmaf(taps.w[k], sx[c + k], acc);
+        so[c] = acc;
+    }
+    __syncwarp();
+    // PE s stopped while holding the sum of output 75-s of its segment (taps 0..s): add it to what is there
+#pragma unroll
+    for (int i = 0; i < RW; ++i) {
+        const int c = kWsSeg1 - 1 - (m * RW + i);
+        yo[c] += Z[i];
     }
 }
 
@@ -411,7 +440,7 @@ conv1d_f32_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, unsig
     }
 }
 
-template <int DESIGN, int Q, int WARPS = DefaultShape1D<DESIGN>::kWarps, int K = DefaultShape1D<DESIGN>::kTiles>
+template <int DESIGN, int Q, int WARPS = DefaultShape1D<DESIGN, Q>::kWarps, int K = DefaultShape1D<DESIGN, Q>::kTiles>
 cudaError_t launch_conv1d_f32_q(const Conv1DArgs &a, const Taps1D &taps, unsigned *status_word, cudaStream_t s)
 {
     using G = Geo1D<DESIGN, WARPS>;
