@@ -12,7 +12,9 @@ to this code.  It shares no code with the CUDA path.
 from .conv import (  # noqa: F401
     build_oracle,
     conv1d_f32,
+    conv1d_f32_strided,
     conv1d_f32_taps_outer,
+    conv2d_f32_strided,
     conv1d_f32_at,
     conv2d_f32,
     conv2d_f32_taps_outer,

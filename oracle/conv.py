@@ -49,6 +49,9 @@ def _load():
             lib.oracle_conv1d_f32_at.argtypes = [_vp, _c_ll, _vp, _c_int, _vp, _c_ll, _vp, _vp]
             lib.oracle_conv2d_f32.argtypes = [_vp, _c_int, _c_int, _c_ll, _vp, _c_int, _c_int,
                                               _vp, _vp, _c_ll]
+            lib.oracle_conv1d_f32_strided.argtypes = [_vp, _c_ll, _vp, _c_int, _c_int, _vp, _vp]
+            lib.oracle_conv2d_f32_strided.argtypes = [_vp, _c_int, _c_int, _c_ll, _vp, _c_int, _c_int,
+                                                      _c_int, _c_int, _vp, _vp, _c_ll]
             lib.oracle_conv2d_f32_taps_outer.argtypes = [_vp, _c_int, _c_int, _c_ll, _vp, _c_int,
                                                          _c_int, _vp, _c_ll]
             lib.oracle_conv2d_f32_at.argtypes = [_vp, _c_int, _c_int, _c_ll, _vp, _c_int, _c_int,
@@ -62,7 +65,8 @@ def _load():
                          "oracle_conv1d_f32_taps_outer", "oracle_conv1d_f32_at",
                          "oracle_conv2d_f32", "oracle_conv2d_f32_taps_outer",
                          "oracle_conv2d_f32_at", "oracle_conv1d_u8s8_s32",
-                         "oracle_conv2d_u8s8_s32", "oracle_conv2d_u8s8_i64"):
+                         "oracle_conv2d_u8s8_s32", "oracle_conv2d_u8s8_i64",
+                         "oracle_conv1d_f32_strided", "oracle_conv2d_f32_strided"):
                 getattr(lib, name).restype = None
             _lib = lib
     return _lib
@@ -97,6 +101,37 @@ def conv1d_f32(x, w, want_scale=True):
     y = np.empty(n - q + 1, dtype=np.float64)
     s = np.empty(n - q + 1, dtype=np.float64) if want_scale else None
     _load().oracle_conv1d_f32(_ptr(x), n, _ptr(w), q, _ptr(y), _ptr(s) if want_scale else None)
+    return y, s
+
+
+def conv1d_f32_strided(x, w, stride, want_scale=True):
+    """Strided Eq. 2, y[c] = sum_q w[q] x[stride*c+q] (Table 2, stride-2 FBS cell) in fp64. Returns (y, S)."""
+    x = _as(x, np.float32, 1)
+    w = _as(w, np.float32, 1)
+    n, q = x.shape[0], w.shape[0]
+    if q < 1 or n < q or stride < 1:
+        raise ValueError("need 1 <= Q <= N and stride >= 1")
+    c = (n - q) // stride + 1
+    y = np.empty(c, dtype=np.float64)
+    s = np.empty(c, dtype=np.float64) if want_scale else None
+    _load().oracle_conv1d_f32_strided(_ptr(x), n, _ptr(w), q, int(stride), _ptr(y),
+                                      _ptr(s) if want_scale else None)
+    return y, s
+
+
+def conv2d_f32_strided(x, w, stride, want_scale=True):
+    """Strided Eq. 3, y[r][c] = sum w[p][q] x[sr*r+p][sc*c+q]; stride = (sr, sc) or one int. Returns (y, S)."""
+    x = _as(x, np.float32, 2)
+    w = _as(w, np.float32, 2)
+    sr, sc = (stride, stride) if np.isscalar(stride) else stride
+    (h, wd), (p, q) = x.shape, w.shape
+    if p < 1 or q < 1 or h < p or wd < q or sr < 1 or sc < 1:
+        raise ValueError("need 1 <= P <= H, 1 <= Q <= W and strides >= 1")
+    oh, ow = (h - p) // sr + 1, (wd - q) // sc + 1
+    y = np.empty((oh, ow), dtype=np.float64)
+    s = np.empty((oh, ow), dtype=np.float64) if want_scale else None
+    _load().oracle_conv2d_f32_strided(_ptr(x), wd, h, wd, _ptr(w), p, q, int(sr), int(sc), _ptr(y),
+                                      _ptr(s) if want_scale else None, ow)
     return y, s
 
 

@@ -104,6 +104,48 @@ void oracle_conv1d_f32_at(const float *x, long long n, const float *w, int q,
     }
 }
 
+/* Strided form of Eq. 2 (the stride-2 FBS cell of Table 2 reads x(2c+q)):
+ * y[c] = sum_q w[q] * x[stride*c + q], c in [0, (n-q)/stride]. s may be NULL. */
+void oracle_conv1d_f32_strided(const float *x, long long n, const float *w, int q,
+                               int stride, double *y, double *s)
+{
+    long long C = (n - q) / stride + 1;
+#pragma omp parallel for schedule(static)
+    for (long long c = 0; c < C; ++c) {
+        double acc = 0.0, mag = 0.0;
+        for (int k = 0; k < q; ++k) {
+            double prod = (double)w[k] * (double)x[(long long)stride * c + k];
+            acc += prod;
+            mag += fabs(prod);
+        }
+        y[c] = acc;
+        if (s) s[c] = mag;
+    }
+}
+
+/* Strided form of Eq. 3: y[r][c] = sum_p sum_q w[p][q] * x[sr*r + p][sc*c + q],
+ * r in [0, (height-p)/sr], c in [0, (width-q)/sc]. s may be NULL. */
+void oracle_conv2d_f32_strided(const float *x, int width, int height, long long x_pitch,
+                               const float *w, int p, int q, int sr, int sc,
+                               double *y, double *s, long long y_pitch)
+{
+    int out_h = (height - p) / sr + 1, out_w = (width - q) / sc + 1;
+#pragma omp parallel for schedule(static)
+    for (int r = 0; r < out_h; ++r)
+        for (int c = 0; c < out_w; ++c) {
+            double acc = 0.0, mag = 0.0;
+            for (int i = 0; i < p; ++i)
+                for (int k = 0; k < q; ++k) {
+                    double prod = (double)w[i * q + k] *
+                                  (double)x[(long long)(sr * r + i) * x_pitch + sc * c + k];
+                    acc += prod;
+                    mag += fabs(prod);
+                }
+            y[(long long)r * y_pitch + c] = acc;
+            if (s) s[(long long)r * y_pitch + c] = mag;
+        }
+}
+
 /* Eq. 3: y[r][c] = sum_p sum_q w[p][q] * x[r+p][c+q].
  * x_pitch / y_pitch are row pitches in elements.  s may be NULL. */
 void oracle_conv2d_f32(const float *x, int width, int height, long long x_pitch,

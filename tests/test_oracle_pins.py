@@ -202,6 +202,72 @@ def test_2d_matches_scipy_correlate2d():
     np.testing.assert_allclose(y, ref, rtol=0, atol=1e-13)
 
 
+# ----------------------------------------------------------------- strided forms
+
+
+@pytest.mark.parametrize("stride", [1, 2, 3])
+def test_1d_strided_is_the_subsampled_numpy_correlation(stride):
+    rng = np.random.default_rng(31)
+    for n, q in [(200, 7), (201, 7), (64, 32), (33, 32), (9, 9)]:
+        x = rng.uniform(-1, 1, n).astype(np.float32)
+        w = rng.uniform(-1, 1, q).astype(np.float32)
+        y, s = oracle.conv1d_f32_strided(x, w, stride)
+        ref = np.correlate(x.astype(np.float64), w.astype(np.float64), mode="valid")[::stride]
+        assert y.shape == ref.shape == ((n - q) // stride + 1,)
+        np.testing.assert_allclose(y, ref, rtol=0, atol=1e-14)
+        ref_s = np.correlate(np.abs(x).astype(np.float64), np.abs(w).astype(np.float64), "valid")[::stride]
+        np.testing.assert_allclose(s, ref_s, rtol=0, atol=1e-14)
+
+
+def test_1d_stride_two_closed_forms():
+    # ramp through a box of Q ones: y[c] = Q*(2c) + Q(Q-1)/2; impulse at tap k: y[c] = x[2c+k]
+    n, q = 101, 6
+    x = np.arange(n, dtype=np.float32)
+    y, _ = oracle.conv1d_f32_strided(x, np.ones(q, np.float32), 2)
+    c = np.arange((n - q) // 2 + 1)
+    np.testing.assert_array_equal(y, q * 2.0 * c + q * (q - 1) / 2)
+    for k in range(q):
+        w = np.zeros(q, np.float32)
+        w[k] = 1
+        y, _ = oracle.conv1d_f32_strided(x, w, 2)
+        np.testing.assert_array_equal(y, x[k::2][:len(c)])
+
+
+def test_1d_stride_two_equals_the_stride_two_fbs_array_of_table_2():
+    from oracle import systolic_sim as sim
+    rng = np.random.default_rng(32)
+    x = _ints(rng, -8, 8, 41)
+    w = _ints(rng, -4, 4, 5)
+    y, _ = oracle.conv1d_f32_strided(x, w, 2)
+    ys, _ = sim.simulate_1d("FBS", x, w, stride=2)
+    np.testing.assert_array_equal(y, np.asarray(ys, dtype=np.float64))
+
+
+@pytest.mark.parametrize("stride", [(1, 1), (2, 2), (2, 1), (1, 2), (3, 2)])
+def test_2d_strided_is_the_subsampled_scipy_correlation(stride):
+    from scipy.signal import correlate2d
+    rng = np.random.default_rng(33)
+    for (h, wd), (p, q) in [((21, 19), (5, 3)), ((20, 18), (3, 5)), ((15, 15), (15, 15)), ((9, 40), (1, 4))]:
+        x = rng.uniform(0, 1, (h, wd)).astype(np.float32)
+        w = rng.uniform(-1, 1, (p, q)).astype(np.float32)
+        y, s = oracle.conv2d_f32_strided(x, w, stride)
+        ref = correlate2d(x.astype(np.float64), w.astype(np.float64), mode="valid")[::stride[0], ::stride[1]]
+        assert y.shape == ref.shape
+        np.testing.assert_allclose(y, ref, rtol=0, atol=1e-13)
+        ref_s = correlate2d(np.abs(x).astype(np.float64), np.abs(w).astype(np.float64), mode="valid")
+        np.testing.assert_allclose(s, ref_s[::stride[0], ::stride[1]], rtol=0, atol=1e-13)
+
+
+def test_2d_stride_two_impulse_and_asymmetry():
+    # an impulse tap at (p0, q0) picks x[2r+p0][2c+q0]: catches a row/column stride swap on a non-square image
+    x = np.arange(11 * 17, dtype=np.float32).reshape(11, 17)
+    w = np.zeros((3, 4), np.float32)
+    w[2, 1] = 1
+    y, _ = oracle.conv2d_f32_strided(x, w, (2, 3))
+    np.testing.assert_array_equal(y, x[2::2, 1::3][:y.shape[0], :y.shape[1]])
+    assert y.shape == ((11 - 3) // 2 + 1, (17 - 4) // 3 + 1)
+
+
 # ----------------------------------------------------------------- integer
 
 
