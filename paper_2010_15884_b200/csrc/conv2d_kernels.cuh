@@ -645,6 +645,8 @@ inline int pick_band_height(int out_h, long long strips_times_batch, int p, int 
     const long long hi = p * q <= 25 ? 64 : 256;
     if (h > hi) h = hi;
     if (h < lo) h = lo;
+    const long long fit = (out_h + 65534LL) / 65535;       // grid.y limit
+    if (h < fit) h = fit;
     return static_cast<int>(h);
 }
 
@@ -688,10 +690,21 @@ cudaError_t launch_conv2d_os_rowpair(const Conv2DArgs &a, const float *w, cudaSt
     return cudaGetLastError();
 }
 
+// Hook for a faster kernel of a (traits, design) pair defined in another header: returns true and sets
+// *err if it launched.  The default does nothing.
+template <typename Tr, int DESIGN, int P, int Q>
+struct FastPath2D {
+    static bool launch(const Conv2DArgs &, const typename Tr::taps_t &, cudaStream_t, cudaError_t *) { return false; }
+};
+
 template <typename Tr, int DESIGN, int P, int Q>
 cudaError_t launch_conv2d_pq(const Conv2DArgs &a, const typename Tr::taps_t &taps, cudaStream_t s)
 {
     if (a.batch > 65535) return cudaErrorInvalidConfiguration;
+    {
+        cudaError_t err = cudaSuccess;
+        if (FastPath2D<Tr, DESIGN, P, Q>::launch(a, taps, s, &err)) return err;
+    }
     if (DESIGN == SYSCONV_WS) {
         // CTAs = width segments x bands of 128 rows x images; segments are multiples of 32 columns and as
         // long as possible (each costs QP-1 fill steps) while still giving a few CTAs per SM
