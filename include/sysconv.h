@@ -116,6 +116,24 @@ int sysconv2d(const void *x_dev, int width, int height, long long x_pitch, long 
               int dtype, int design, void *stream);
 
 /*
+ * Strided forms: y(c) = sum_q x(stride*c + q) w(q) with (n-q)/stride + 1 outputs per signal (the stride-2
+ * FBS design of Table 2), and y(r, c) = sum_p sum_q x(stride_r*r + p, stride_c*c + q) w(p, q) with
+ * ((height-p)/stride_r + 1) x ((width-q)/stride_c + 1) outputs per image (Section 5 runs the strided
+ * design row by row).  All other arguments as for sysconv1d / sysconv2d.
+ * Stride 1 is the unstrided call.  Stride 2 (both directions in 2-D) is built for fp32 data, the
+ * SYSCONV_OS and SYSCONV_IS designs, q <= 32 in 1-D and p, q <= 7 in 2-D; every other combination returns
+ * SYSCONV_EUNSUPPORTED (strides below 1: SYSCONV_EINVAL).
+ */
+int sysconv1d_strided(const void *x_dev, long long n, long long x_batch_stride,
+                      const void *w_host, int q, int stride,
+                      void *y_dev, long long y_batch_stride, int batch,
+                      int dtype, int design, void *stream);
+int sysconv2d_strided(const void *x_dev, int width, int height, long long x_pitch, long long x_batch_stride,
+                      const void *w_host, int q, int p, int stride_c, int stride_r,
+                      void *y_dev, long long y_pitch, long long y_batch_stride, int batch,
+                      int dtype, int design, void *stream);
+
+/*
  * The same two operations for callers whose data lives in HOST memory
  * (densely packed: pitch = row length, batch stride = array size).  The call
  * enqueues the host-to-device copy of x into the caller's device workspace,

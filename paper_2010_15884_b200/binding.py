@@ -49,6 +49,11 @@ def load_library():
     lib.sysconv2d.restype = _c_int
     lib.sysconv2d.argtypes = [_vp, _c_int, _c_int, _c_ll, _c_ll, _vp, _c_int, _c_int, _vp, _c_ll, _c_ll,
                               _c_int, _c_int, _c_int, _vp]
+    lib.sysconv1d_strided.restype = _c_int
+    lib.sysconv1d_strided.argtypes = [_vp, _c_ll, _c_ll, _vp, _c_int, _c_int, _vp, _c_ll, _c_int, _c_int, _c_int, _vp]
+    lib.sysconv2d_strided.restype = _c_int
+    lib.sysconv2d_strided.argtypes = [_vp, _c_int, _c_int, _c_ll, _c_ll, _vp, _c_int, _c_int, _c_int, _c_int, _vp,
+                                      _c_ll, _c_ll, _c_int, _c_int, _c_int, _vp]
     lib.sysconv1d_host_workspace_bytes.restype = _c_ll
     lib.sysconv1d_host_workspace_bytes.argtypes = [_c_ll, _c_int, _c_int, _c_int]
     lib.sysconv2d_host_workspace_bytes.restype = _c_ll
@@ -135,6 +140,21 @@ def sysconv2d(x_ptr, width, height, x_pitch, x_batch_stride, w_host, q, p, y_ptr
                              _vp(stream_ptr)))
 
 
+def sysconv1d_strided(x_ptr, n, x_batch_stride, w_host, q, stride, y_ptr, y_batch_stride, batch, dtype, design,
+                      stream_ptr):
+    lib = load_library()
+    return int(lib.sysconv1d_strided(_vp(x_ptr), n, x_batch_stride, w_host.ctypes.data_as(_vp), q, stride,
+                                     _vp(y_ptr), y_batch_stride, batch, dtype, design, _vp(stream_ptr)))
+
+
+def sysconv2d_strided(x_ptr, width, height, x_pitch, x_batch_stride, w_host, q, p, stride_c, stride_r, y_ptr,
+                      y_pitch, y_batch_stride, batch, dtype, design, stream_ptr):
+    lib = load_library()
+    return int(lib.sysconv2d_strided(_vp(x_ptr), width, height, x_pitch, x_batch_stride,
+                                     w_host.ctypes.data_as(_vp), q, p, stride_c, stride_r, _vp(y_ptr), y_pitch,
+                                     y_batch_stride, batch, dtype, design, _vp(stream_ptr)))
+
+
 def host_workspace_bytes(shape, filt, dtype=F32):
     """Device workspace the *_host entry points need. shape = (n,) | (batch, n) | (h, w) handled by caller."""
     lib = load_library()
@@ -210,8 +230,8 @@ def _dtype_of(x):
     raise TypeError("x must be float32 or uint8, got %s" % x.dtype)
 
 
-def conv1d(x, w, design=OS, out=None, stream=None):
-    """y[b, c] = sum_k w[k] x[b, c+k] on CUDA tensors. x: (n,) or (batch, n), contiguous rows."""
+def conv1d(x, w, design=OS, out=None, stream=None, stride=1):
+    """y[b, c] = sum_k w[k] x[b, stride*c+k] on CUDA tensors. x: (n,) or (batch, n), contiguous rows."""
     import torch
     if not x.is_cuda:
         raise SysconvError(-1, "conv1d (x is not a CUDA tensor; there is no CPU path)")
@@ -223,21 +243,22 @@ def conv1d(x, w, design=OS, out=None, stream=None):
     taps = _host_taps(w, dtype, 1)
     batch, n = x2.shape
     q = taps.shape[0]
+    n_out = (n - q) // stride + 1 if n >= q else 0
     if out is None:
-        out = torch.empty((batch, n - q + 1) if n >= q else (batch, 0), dtype=out_dtype, device=x.device)
+        out = torch.empty((batch, n_out), dtype=out_dtype, device=x.device)
         y2 = out
     else:
         y2 = out.unsqueeze(0) if out.dim() == 1 else out
-    st = sysconv1d(x2.data_ptr(), n, x2.stride(0) if batch > 1 else n, taps, q, y2.data_ptr(),
-                   y2.stride(0) if batch > 1 else max(n - q + 1, 0), batch, dtype, _design(design),
-                   _stream_ptr(stream))
+    st = sysconv1d_strided(x2.data_ptr(), n, x2.stride(0) if batch > 1 else n, taps, q, stride, y2.data_ptr(),
+                           y2.stride(0) if batch > 1 else n_out, batch, dtype, _design(design),
+                           _stream_ptr(stream))
     if st != 0:
-        raise SysconvError(st, "sysconv1d")
+        raise SysconvError(st, "sysconv1d" if stride == 1 else "sysconv1d_strided")
     return out.squeeze(0) if (squeeze and out.dim() == 2) else out
 
 
-def conv2d(x, w, design=OS, out=None, stream=None):
-    """y[b, r, c] = sum_p sum_q w[p, q] x[b, r+p, c+q] on CUDA tensors. x: (h, w) or (batch, h, w)."""
+def conv2d(x, w, design=OS, out=None, stream=None, stride=1):
+    """y[b, r, c] = sum_p sum_q w[p, q] x[b, stride*r+p, stride*c+q] on CUDA tensors. x: (h, w) or (batch, h, w)."""
     import torch
     if not x.is_cuda:
         raise SysconvError(-1, "conv2d (x is not a CUDA tensor; there is no CPU path)")
@@ -250,13 +271,15 @@ def conv2d(x, w, design=OS, out=None, stream=None):
     batch, h, wd = x3.shape
     p, q = taps.shape
     if out is None:
-        out = torch.empty((batch, max(h - p + 1, 0), max(wd - q + 1, 0)), dtype=out_dtype, device=x.device)
+        oh = (h - p) // stride + 1 if h >= p else 0
+        ow = (wd - q) // stride + 1 if wd >= q else 0
+        out = torch.empty((batch, oh, ow), dtype=out_dtype, device=x.device)
         y3 = out
     else:
         y3 = out.unsqueeze(0) if out.dim() == 2 else out
-    st = sysconv2d(x3.data_ptr(), wd, h, x3.stride(1), x3.stride(0) if batch > 1 else 0, taps, q, p,
-                   y3.data_ptr(), y3.stride(1), y3.stride(0) if batch > 1 else 0, batch, dtype,
-                   _design(design), _stream_ptr(stream))
+    st = sysconv2d_strided(x3.data_ptr(), wd, h, x3.stride(1), x3.stride(0) if batch > 1 else 0, taps, q, p,
+                           stride, stride, y3.data_ptr(), y3.stride(1), y3.stride(0) if batch > 1 else 0, batch,
+                           dtype, _design(design), _stream_ptr(stream))
     if st != 0:
-        raise SysconvError(st, "sysconv2d")
+        raise SysconvError(st, "sysconv2d" if stride == 1 else "sysconv2d_strided")
     return out.squeeze(0) if (squeeze and out.dim() == 3) else out

@@ -175,6 +175,69 @@ int sysconv1d(const void *x_dev, long long n, long long x_batch_stride, const vo
     return dispatch2d(a, w_host, q, 1, dtype, design, s);
 }
 
+int sysconv1d_strided(const void *x_dev, long long n, long long x_batch_stride, const void *w_host, int q, int stride,
+                      void *y_dev, long long y_batch_stride, int batch, int dtype, int design, void *stream)
+{
+    using namespace sysconv;
+    if (stride < 1) return SYSCONV_EINVAL;
+    if (stride == 1)
+        return sysconv1d(x_dev, n, x_batch_stride, w_host, q, y_dev, y_batch_stride, batch, dtype, design, stream);
+    if (!x_dev || !y_dev || !w_host) return SYSCONV_EINVAL;
+    if (!valid_enums(dtype, design)) return SYSCONV_EINVAL;
+    if (q < 1 || n < q || batch < 1) return SYSCONV_EINVAL;
+    const long long n_out = (n - q) / stride + 1;
+    if (batch > 1 && (x_batch_stride < n || y_batch_stride < n_out)) return SYSCONV_EINVAL;
+    if (batch == 1) { x_batch_stride = n; y_batch_stride = n_out; }
+    const unsigned long long x_bytes = ((unsigned long long)(batch - 1) * x_batch_stride + n) * in_elt_bytes(dtype);
+    const unsigned long long y_bytes = ((unsigned long long)(batch - 1) * y_batch_stride + n_out) * 4ull;
+    if (overlaps(x_dev, x_bytes, y_dev, y_bytes)) return SYSCONV_EINVAL;
+    if (stride != 2 || dtype != SYSCONV_F32 || q > kMaxQ1) return SYSCONV_EUNSUPPORTED;
+    if (design != SYSCONV_OS && design != SYSCONV_IS) return SYSCONV_EUNSUPPORTED;
+    Conv1DArgs a;
+    a.x = x_dev; a.y = y_dev; a.n = n; a.n_out = n_out;
+    a.x_bstride = x_batch_stride; a.y_bstride = y_batch_stride; a.batch = batch;
+    int launches = 0;
+    const DeviceInfo *d = device_info();
+    if (!d) return SYSCONV_ECUDA;
+    const cudaError_t err = launch_conv1d_f32_stride2(design, a, static_cast<const float *>(w_host), q, d->status_word,
+                                                      static_cast<cudaStream_t>(stream), &launches);
+    return finish(err, launches);
+}
+
+int sysconv2d_strided(const void *x_dev, int width, int height, long long x_pitch, long long x_batch_stride,
+                      const void *w_host, int q, int p, int stride_c, int stride_r, void *y_dev, long long y_pitch,
+                      long long y_batch_stride, int batch, int dtype, int design, void *stream)
+{
+    using namespace sysconv;
+    if (stride_c < 1 || stride_r < 1) return SYSCONV_EINVAL;
+    if (stride_c == 1 && stride_r == 1)
+        return sysconv2d(x_dev, width, height, x_pitch, x_batch_stride, w_host, q, p, y_dev, y_pitch, y_batch_stride,
+                         batch, dtype, design, stream);
+    if (!x_dev || !y_dev || !w_host) return SYSCONV_EINVAL;
+    if (!valid_enums(dtype, design)) return SYSCONV_EINVAL;
+    if (q < 1 || p < 1 || width < q || height < p || batch < 1) return SYSCONV_EINVAL;
+    const int out_w = (width - q) / stride_c + 1, out_h = (height - p) / stride_r + 1;
+    if (x_pitch < width || y_pitch < out_w) return SYSCONV_EINVAL;
+    const long long x_img = (long long)(height - 1) * x_pitch + width;
+    const long long y_img = (long long)(out_h - 1) * y_pitch + out_w;
+    if (batch > 1 && (x_batch_stride < x_img || y_batch_stride < y_img)) return SYSCONV_EINVAL;
+    if (batch == 1) { x_batch_stride = x_img; y_batch_stride = y_img; }
+    const unsigned long long x_bytes = ((unsigned long long)(batch - 1) * x_batch_stride + x_img) * in_elt_bytes(dtype);
+    const unsigned long long y_bytes = ((unsigned long long)(batch - 1) * y_batch_stride + y_img) * 4ull;
+    if (overlaps(x_dev, x_bytes, y_dev, y_bytes)) return SYSCONV_EINVAL;
+    if (stride_c != 2 || stride_r != 2 || dtype != SYSCONV_F32) return SYSCONV_EUNSUPPORTED;
+    if (design != SYSCONV_OS && design != SYSCONV_IS) return SYSCONV_EUNSUPPORTED;
+    Conv2DArgs a;
+    a.x = x_dev; a.y = y_dev;
+    a.width = width; a.height = height; a.out_w = out_w; a.out_h = out_h;
+    a.x_pitch = x_pitch; a.y_pitch = y_pitch;
+    a.x_bstride = x_batch_stride; a.y_bstride = y_batch_stride; a.batch = batch;
+    int launches = 0;
+    const cudaError_t err = launch_conv2d_f32_stride2(design, a, static_cast<const float *>(w_host), q, p,
+                                                      static_cast<cudaStream_t>(stream), &launches);
+    return finish(err, launches);
+}
+
 int sysconv2d(const void *x_dev, int width, int height, long long x_pitch, long long x_batch_stride,
               const void *w_host, int q, int p, void *y_dev, long long y_pitch, long long y_batch_stride,
               int batch, int dtype, int design, void *stream)

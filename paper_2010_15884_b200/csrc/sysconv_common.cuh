@@ -85,6 +85,12 @@ cudaError_t launch_conv1d_f32_ws(const Conv1DArgs &a, const float *w, int q, uns
 cudaError_t launch_conv1d_f32_other(int design, const Conv1DArgs &a, const float *w, int q, unsigned *status_word,
                                     cudaStream_t s, int *launches);
 
+// stride-2 forms (design = SYSCONV_OS or SYSCONV_IS); a.n_out / a.out_w, a.out_h are the strided output sizes
+cudaError_t launch_conv1d_f32_stride2(int design, const Conv1DArgs &a, const float *w, int q, unsigned *status_word,
+                                      cudaStream_t s, int *launches);
+cudaError_t launch_conv2d_f32_stride2(int design, const Conv2DArgs &a, const float *w, int q, int p, cudaStream_t s,
+                                      int *launches);
+
 cudaError_t launch_conv2d_f32_os(const Conv2DArgs &a, const float *w, int q, int p, cudaStream_t s, int *launches);
 cudaError_t launch_conv2d_f32_is(const Conv2DArgs &a, const float *w, int q, int p, cudaStream_t s, int *launches);
 cudaError_t launch_conv2d_f32_ws(const Conv2DArgs &a, const float *w, int q, int p, cudaStream_t s, int *launches);

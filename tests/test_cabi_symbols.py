@@ -25,7 +25,7 @@ def _declared_functions():
 
 def test_header_declares_the_expected_entry_points():
     names = _declared_functions()
-    for must in ("sysconv1d", "sysconv2d", "sysconv1d_host", "sysconv2d_host", "sysconv_status_string",
+    for must in ("sysconv1d", "sysconv2d", "sysconv1d_strided", "sysconv2d_strided", "sysconv1d_host", "sysconv2d_host", "sysconv_status_string",
                  "sysconv_design_name", "sysconv_version", "sysconv_launch_count"):
         assert must in names
 
@@ -73,3 +73,26 @@ def test_argument_validation_needs_no_gpu(lib):
     assert lib.sysconv1d_host_workspace_bytes(100, 4, 2, b.F32) == 1024 + 1024
     assert lib.sysconv1d_host_workspace_bytes(3, 4, 1, b.F32) == -1
     assert lib.sysconv2d_host_workspace_bytes(10, 10, 3, 3, 1, b.U8S8_S32) == 256 + 256
+
+
+def test_strided_argument_validation_needs_no_gpu(lib):
+    import numpy as np
+    from paper_2010_15884_b200 import binding as b
+    w = np.ones(4, np.float32)
+    w2 = np.ones((3, 3), np.float32)
+    wi = np.ones((3, 3), np.int8)
+    x, y = 0x10000, 0x90000000
+    assert b.sysconv1d_strided(x, 100, 100, w, 4, 0, y, 49, 1, b.F32, b.OS, 0) == 1        # stride < 1
+    assert b.sysconv1d_strided(0, 100, 100, w, 4, 2, y, 49, 1, b.F32, b.OS, 0) == 1        # null x
+    assert b.sysconv1d_strided(x, 3, 3, w, 4, 2, y, 1, 1, b.F32, b.OS, 0) == 1             # n < q
+    assert b.sysconv1d_strided(x, 100, 100, w, 4, 2, y, 40, 2, b.F32, b.OS, 0) == 1        # y batch stride < n_out
+    assert b.sysconv1d_strided(x, 100, 100, w, 4, 3, y, 33, 1, b.F32, b.OS, 0) == 2        # stride 3: not built
+    assert b.sysconv1d_strided(x, 100, 100, w, 4, 2, y, 49, 1, b.F32, b.WS, 0) == 2        # WS: not built
+    assert b.sysconv1d_strided(x, 100, 100, w, 4, 2, y, 49, 1, b.U8S8_S32, b.OS, 0) == 2   # integer: not built
+    assert b.sysconv2d_strided(x, 64, 64, 64, 0, w2, 3, 3, 2, 0, y, 31, 0, 1, b.F32, b.OS, 0) == 1     # stride_r < 1
+    assert b.sysconv2d_strided(x, 64, 64, 64, 0, w2, 3, 3, 2, 2, y, 30, 0, 1, b.F32, b.OS, 0) == 1     # y_pitch < out_w
+    assert b.sysconv2d_strided(x, 64, 64, 64, 0, w2, 3, 3, 2, 1, y, 31, 0, 1, b.F32, b.OS, 0) == 2     # mixed strides
+    assert b.sysconv2d_strided(x, 64, 64, 64, 0, w2, 3, 3, 2, 2, y, 31, 0, 1, b.F32, b.WS, 0) == 2     # WS: not built
+    assert b.sysconv2d_strided(x, 64, 64, 64, 0, wi, 3, 3, 2, 2, y, 31, 0, 1, b.U8S8_S32, b.IS, 0) == 2
+    w9 = np.ones((9, 9), np.float32)
+    assert b.sysconv2d_strided(x, 64, 64, 64, 0, w9, 9, 9, 2, 2, y, 28, 0, 1, b.F32, b.OS, 0) == 2     # beyond 7 x 7

@@ -390,6 +390,146 @@ def test_2d_non_finite_inputs_stay_inside_their_windows(cuda_device, design, pq)
     assert (np.abs(y[loose] - y_ref[loose]) <= TOL * s_ref[loose]).all()
 
 
+# ------------------------------------------------------------------------ stride 2 (Table 2, cell 6)
+
+STRIDED_DESIGNS = [B.OS, B.IS]
+
+
+@pytest.mark.parametrize("design", STRIDED_DESIGNS, ids=_ids)
+@pytest.mark.parametrize("q", [1, 2, 3, 4, 5, 7, 8, 15, 16, 31, 32])
+def test_1d_stride2_filter_sizes(cuda_device, design, q):
+    n = 3 * 2432 + 1216 + 37          # several CTA tiles, one ragged
+    x, ws = inputs.gen_1d_f32(n, [q], seed=300 + q)
+    y = B.conv1d(torch.from_numpy(x).to(cuda_device), ws[q], design, stride=2)
+    torch.cuda.synchronize()
+    y_ref, s_ref = oracle.conv1d_f32_strided(x, ws[q], 2)
+    assert y.shape == y_ref.shape
+    assert_close_f32(y.cpu().numpy(), y_ref, s_ref, "stride 2, q=%d" % q)
+
+
+@pytest.mark.parametrize("design", STRIDED_DESIGNS, ids=_ids)
+@pytest.mark.parametrize("n", [5, 6, 7, 8, 303, 304, 305, 607, 608, 609, 639, 640, 641, 1216, 1217, 1247, 1248, 1249,
+                               2431, 2432, 2433, 2463, 2464, 2465, 4864 + 33])
+def test_1d_stride2_lengths_around_tile_edges(cuda_device, design, n):
+    q = 5
+    x, ws = inputs.gen_1d_f32(n, [q], seed=400 + n % 97)
+    y = B.conv1d(torch.from_numpy(x).to(cuda_device), ws[q], design, stride=2)
+    torch.cuda.synchronize()
+    y_ref, s_ref = oracle.conv1d_f32_strided(x, ws[q], 2)
+    assert y.shape == y_ref.shape
+    assert_close_f32(y.cpu().numpy(), y_ref, s_ref, "stride 2, n=%d" % n)
+
+
+@pytest.mark.parametrize("design", STRIDED_DESIGNS, ids=_ids)
+def test_1d_stride2_batch_unaligned_and_canaries(cuda_device, design):
+    q, n, batch = 9, 7001, 3
+    x, ws = inputs.gen_1d_f32(n * batch, [q], seed=77)
+    x = x.reshape(batch, n)
+    n_out = (n - q) // 2 + 1
+    for x_off, y_off, xs, ys in [(0, 0, n, n_out), (1, 3, n + 3, n_out + 5), (4, 4, n + 4, n_out + 4)]:
+        xb = torch.zeros(x_off + batch * xs + 8, dtype=torch.float32, device=cuda_device)
+        yb = torch.full((y_off + batch * ys + 8,), CANARY, dtype=torch.float32, device=cuda_device)
+        xb[x_off: x_off + batch * xs].view(batch, xs)[:, :n] = torch.from_numpy(x).to(cuda_device)
+        st = B.sysconv1d_strided(xb.data_ptr() + 4 * x_off, n, xs, ws[q], q, 2, yb.data_ptr() + 4 * y_off, ys, batch,
+                                 B.F32, design, torch.cuda.current_stream().cuda_stream)
+        assert st == 0, B.status_string(st)
+        torch.cuda.synchronize()
+        yh = yb.cpu().numpy()
+        body = yh[y_off: y_off + batch * ys].reshape(batch, ys)
+        assert (body[:, n_out:] == CANARY).all() and (yh[:y_off] == CANARY).all()
+        assert (yh[y_off + batch * ys:] == CANARY).all()
+        for b in range(batch):
+            y_ref, s_ref = oracle.conv1d_f32_strided(x[b], ws[q], 2)
+            assert_close_f32(body[b, :n_out], y_ref, s_ref, "signal %d" % b)
+
+
+def test_1d_stride2_large_sampled(cuda_device):
+    n, q = (1 << 24) + 3, 16
+    x, ws = inputs.gen_1d_f32(n, [q], seed=9)
+    xd = torch.from_numpy(x).to(cuda_device)
+    rng = np.random.default_rng(5)
+    n_out = (n - q) // 2 + 1
+    pos = np.unique(np.concatenate([rng.integers(0, n_out, 4000), np.arange(64), np.arange(n_out - 64, n_out)]))
+    y_ref, s_ref = oracle.conv1d_f32_at(x, ws[q], 2 * pos)
+    for design in STRIDED_DESIGNS:
+        y = B.conv1d(xd, ws[q], design, stride=2)
+        torch.cuda.synchronize()
+        assert y.numel() == n_out
+        assert_close_f32(y.cpu().numpy()[pos], y_ref, s_ref, "sampled, %s" % B.DESIGN_NAMES[design])
+
+
+def run_2d_s2(x_np, w_np, design, device, x_pitch=None, y_pitch=None, x_off=0, y_off=0):
+    batch, h, wd = x_np.shape
+    p, q = w_np.shape
+    oh, ow = (h - p) // 2 + 1, (wd - q) // 2 + 1
+    x_pitch = x_pitch or wd
+    y_pitch = y_pitch or ow
+    xb = torch.zeros(x_off + batch * h * x_pitch + 16, dtype=torch.float32, device=device)
+    yb = torch.full((y_off + batch * oh * y_pitch + 64,), CANARY, dtype=torch.float32, device=device)
+    xb[x_off: x_off + batch * h * x_pitch].view(batch, h, x_pitch)[:, :, :wd] = torch.from_numpy(x_np).to(device)
+    st = B.sysconv2d_strided(xb.data_ptr() + 4 * x_off, wd, h, x_pitch, h * x_pitch, np.ascontiguousarray(w_np), q, p,
+                             2, 2, yb.data_ptr() + 4 * y_off, y_pitch, oh * y_pitch, batch, B.F32, design,
+                             torch.cuda.current_stream().cuda_stream)
+    assert st == 0, B.status_string(st)
+    torch.cuda.synchronize()
+    yh = yb.cpu().numpy()
+    body = yh[y_off: y_off + batch * oh * y_pitch].reshape(batch, oh, y_pitch)
+    assert (body[:, :, ow:] == CANARY).all(), "write into the pitch padding"
+    assert (yh[:y_off] == CANARY).all() and (yh[y_off + batch * oh * y_pitch:] == CANARY).all()
+    return body[:, :, :ow].copy()
+
+
+def check_2d_s2(x_np, w_np, design, device, **kw):
+    y = run_2d_s2(x_np, w_np, design, device, **kw)
+    for b in range(x_np.shape[0]):
+        y_ref, s_ref = oracle.conv2d_f32_strided(x_np[b], w_np, 2)
+        assert y[b].shape == y_ref.shape
+        assert_close_f32(y[b], y_ref, s_ref, "image %d" % b)
+
+
+@pytest.mark.parametrize("design", STRIDED_DESIGNS, ids=_ids)
+@pytest.mark.parametrize("pq", [(p, q) for p in range(1, 8) for q in range(1, 8)], ids=lambda f: "%dx%d" % f)
+def test_2d_stride2_all_filter_shapes(cuda_device, design, pq):
+    x, ws = inputs.gen_2d_f32(533, 61, [pq], seed=500 + 8 * pq[0] + pq[1], batch=2)
+    check_2d_s2(x, ws[pq], design, cuda_device)
+
+
+@pytest.mark.parametrize("design", STRIDED_DESIGNS, ids=_ids)
+@pytest.mark.parametrize("hw", [(0, 0), (1, 0), (0, 1), (1, 1), (2, 3), (9, 239), (10, 240), (11, 241), (12, 247),
+                                (13, 248), (14, 249), (5, 255), (6, 256), (7, 257), (8, 1000)])
+@pytest.mark.parametrize("pq", [(3, 3), (2, 5), (7, 7)], ids=lambda f: "%dx%d" % f)
+def test_2d_stride2_sizes_around_strip_and_band_edges(cuda_device, design, pq, hw):
+    p, q = pq
+    h, wd = p + hw[0], q + hw[1]
+    x, ws = inputs.gen_2d_f32(wd, h, [pq], seed=600 + h + wd, batch=1)
+    check_2d_s2(x, ws[pq], design, cuda_device)
+
+
+@pytest.mark.parametrize("design", STRIDED_DESIGNS, ids=_ids)
+def test_2d_stride2_pitch_offsets_and_tall_image(cuda_device, design):
+    x, ws = inputs.gen_2d_f32(301, 75, [(3, 3), (5, 4)], seed=71, batch=2)
+    for pq in [(3, 3), (5, 4)]:
+        check_2d_s2(x, ws[pq], design, cuda_device, x_pitch=307, y_pitch=155, x_off=1, y_off=1)
+        check_2d_s2(x, ws[pq], design, cuda_device, x_pitch=304, y_pitch=152, x_off=4, y_off=4)
+    x, ws = inputs.gen_2d_f32(70, 2100, [(7, 3)], seed=72, batch=1)
+    check_2d_s2(x, ws[(7, 3)], design, cuda_device)
+
+
+def test_2d_stride2_full_hd_sampled(cuda_device):
+    x, ws = inputs.gen_2d_f32(1920, 1080, [(5, 5)], seed=73, batch=1)
+    xd = torch.from_numpy(x).to(cuda_device)
+    rng = np.random.default_rng(6)
+    oh, ow = (1080 - 5) // 2 + 1, (1920 - 5) // 2 + 1
+    rows = np.concatenate([rng.integers(0, oh, 3000), [0, 0, oh - 1, oh - 1]])
+    cols = np.concatenate([rng.integers(0, ow, 3000), [0, ow - 1, 0, ow - 1]])
+    y_ref, s_ref = oracle.conv2d_f32_at(x[0], ws[(5, 5)], 2 * rows, 2 * cols)
+    for design in STRIDED_DESIGNS:
+        y = B.conv2d(xd, ws[(5, 5)], design, stride=2)
+        torch.cuda.synchronize()
+        assert tuple(y.shape) == (1, oh, ow)
+        assert_close_f32(y.cpu().numpy()[0][rows, cols], y_ref, s_ref, "sampled, %s" % B.DESIGN_NAMES[design])
+
+
 # ------------------------------------------------------------------------ integer
 
 
@@ -410,6 +550,24 @@ def test_2d_u8_shapes_and_extremes(cuda_device, design, pq):
     xm = np.full((1, 40, 150), 255, np.uint8)
     for v in (8, -8):
         check_2d(xm, np.full(pq, v, np.int8), design, cuda_device)
+
+
+@pytest.mark.parametrize("pq", [(1, 1), (3, 3), (5, 5), (7, 7), (7, 15), (8, 15), (15, 15), (9, 2), (4, 13), (12, 8)],
+                         ids=lambda f: "%dx%d" % f)
+def test_2d_u8_os_packed_rows(cuda_device, pq):
+    """Rows that start 16-byte aligned take the packed four-taps-per-step kernel: several strips, a ragged
+    right edge, pitch padding, unaligned outputs, and the extreme pixel/tap values."""
+    p, q = pq
+    x, ws = inputs.gen_2d_u8s8(1101, 41, [pq], seed=90 + p + q, batch=2)
+    check_2d(x, ws[pq], B.OS, cuda_device, x_pitch=1104)
+    check_2d(x, ws[pq], B.OS, cuda_device, x_pitch=1120, y_pitch=1103, y_off=3)
+    check_2d(x[:, :, :1040], ws[pq], B.OS, cuda_device)
+    check_2d(x[:, :, :528], ws[pq], B.OS, cuda_device, x_pitch=528)
+    xm = np.full((1, 33, 160), 255, np.uint8)
+    for v in (127, -128):
+        check_2d(xm, np.full(pq, v, np.int8), B.OS, cuda_device)
+    wmix = np.where((np.arange(p * q).reshape(p, q) % 2) == 0, 127, -128).astype(np.int8)
+    check_2d(x[:1, :, :512], wmix, B.OS, cuda_device)
 
 
 @pytest.mark.parametrize("design", DESIGNS, ids=_ids)
