@@ -39,6 +39,9 @@ sys.path.insert(0, ROOT)
 HBM_FALLBACK_GBS = 6650.0
 SM_COUNT = 148
 FP32_LANES_PER_SM = 128
+# dp4a issues on 64 lanes per clock per SM on B200 (measured: 63.5, the same as the 32-bit integer multiply-add)
+# and does four 8-bit multiply-adds per lane: the ALU roofline of the uint8 x int8 path
+INT8_DOT_MACS_PER_SM = 256
 NAMES = {0: "WS", 1: "OS", 2: "IS"}
 
 
@@ -113,9 +116,11 @@ class ClockSampler:
 class Case:
     """One kernel launch of a workload: a (filter, design) pair on resident device buffers."""
 
-    def __init__(self, cfg, label, design, launch, n_out, alg_bytes, macs):
+    def __init__(self, cfg, label, design, launch, n_out, alg_bytes, macs, mac_lanes=None):
         self.cfg, self.label, self.design, self.launch = cfg, label, design, launch
         self.n_out, self.alg_bytes, self.macs = n_out, alg_bytes, macs
+        # multiply-adds per clock per SM of the plain (non-tensor) datapath this case runs on
+        self.mac_lanes = mac_lanes or FP32_LANES_PER_SM
         self.times_ms = []
 
 
@@ -168,14 +173,62 @@ def build_cases(cfg_id, device, designs=(0, 1, 2), scale=None):
                           oh * y_pitch, batch, dtype, d, stream))
         keep.append(yd)
         for d in designs:
-            cases.append(Case(cfg_id, label, d, mk(d), n_out, alg, macs))
+            cases.append(Case(cfg_id, label, d, mk(d), n_out, alg, macs,
+                              INT8_DOT_MACS_PER_SM if kind == "2d_u8s8" else None))
+    return cases, keep
+
+
+def build_strided_cases(device):
+    """Stride-2 forms (Table 2, cell 6) at the sizes of configurations 2 and 5: OS and IS designs."""
+    import torch
+    from paper_2010_15884_b200 import binding as B
+    from paper_2010_15884_b200 import inputs
+    stream = torch.cuda.current_stream().cuda_stream
+    cases, keep = [], []
+
+    def checked(call, *cargs):
+        def run():
+            st = call(*cargs)
+            if st != 0:
+                raise B.SysconvError(st, call.__name__)
+        return run
+
+    x, ws = inputs.make_config(2)
+    xd = torch.from_numpy(x).to(device)
+    keep.append(xd)
+    n = x.shape[0]
+    for q, w in ws.items():
+        n_out = (n - q) // 2 + 1
+        yd = torch.empty(n_out, dtype=torch.float32, device=device)
+        keep += [w, yd]
+        for d in (B.OS, B.IS):
+            cases.append(Case("2/stride2", "Q=%d" % q, d,
+                              checked(B.sysconv1d_strided, xd.data_ptr(), n, n, w, q, 2, yd.data_ptr(), n_out, 1,
+                                      B.F32, d, stream), n_out, 4 * n + 4 * n_out, n_out * q))
+    x, ws = inputs.make_config(5, dict(filters=[3]))
+    x2 = torch.from_numpy(x).to(device)
+    keep.append(x2)
+    batch, h, wd = x.shape
+    rng = np.random.default_rng(11)
+    for k in (3, 7):
+        w = rng.normal(0, 1.0 / k, (k, k)).astype(np.float32)
+        oh, ow = (h - k) // 2 + 1, (wd - k) // 2 + 1
+        y_pitch = (ow + 3) // 4 * 4
+        yd = torch.empty((batch, oh, y_pitch), dtype=torch.float32, device=device)
+        keep += [w, yd]
+        n_out = batch * oh * ow
+        for d in (B.OS, B.IS):
+            cases.append(Case("5/stride2", "%dx%d" % (k, k), d,
+                              checked(B.sysconv2d_strided, x2.data_ptr(), wd, h, wd, h * wd, w, k, k, 2, 2,
+                                      yd.data_ptr(), y_pitch, oh * y_pitch, batch, B.F32, d, stream),
+                              n_out, x.size * 4 + 4 * n_out, n_out * k * k))
     return cases, keep
 
 
 def roofline_time_s(case, hbm_gbs, sm_mhz):
     """max(bytes / HBM bandwidth, MACs / plain-ALU MAC rate) for one launch."""
     t_mem = case.alg_bytes / (hbm_gbs * 1e9)
-    mac_rate = SM_COUNT * FP32_LANES_PER_SM * sm_mhz * 1e6
+    mac_rate = SM_COUNT * case.mac_lanes * sm_mhz * 1e6
     t_alu = case.macs / mac_rate
     return max(t_mem, t_alu), ("hbm" if t_mem >= t_alu else "alu")
 
@@ -539,6 +592,11 @@ def all_config_detail(device, hbm_gbs, peak_kind, sm_max, skip, reps):
         rows += detail_rows(cases, hbm_gbs, peak_kind, sm_max)
         del cases, keep
         torch.cuda.empty_cache()
+    cases, keep = build_strided_cases(device)
+    time_cases_individually(cases, 3, reps, None)
+    rows += detail_rows(cases, hbm_gbs, peak_kind, sm_max)
+    del cases, keep
+    torch.cuda.empty_cache()
     return rows
 
 
