@@ -109,13 +109,19 @@ __device__ __forceinline__ void os_pass_1d(const float *sx, float *so, const Tap
 // (one shuffle per step).  The partial sums of two neighbouring PEs c (even) and c+1 share a 64-bit
 // register pair, and ONE packed fp32x2 FMA (fma.rn.f32x2, sm_100) serves both: the input that PE c uses
 // with tap t at step t is the input PE c+1 used with tap t-1, so the multiplicand is (x, x) and the
-// multiplier the tap pair (w(t), w(t-1)), which comes straight from the kernel parameters as a
-// uniform-register pair.  Q+1 steps of R1/2 packed FMAs replace Q steps of R1 scalar ones: about half
+// multiplier the tap pair (w(t), w(t-1)), which comes straight from the kernel parameters as an aligned
+// uniform-register pair (the pairs are laid out by the launcher: built in the kernel from the plain tap
+// array they cost almost one uniform move per packed FMA).  Q+1 steps of R1/2 packed FMAs replace Q steps of R1 scalar ones: about half
 // the issue slots per MAC (the scalar form is issue-bound at Q = 32).  In the first and the last step
 // only one PE of each pair has a tap: those two steps use scalar FMAs, so that no input outside an
 // output's window ever enters its sum (a zero tap times a non-finite input would).
+struct Taps1DPairs {
+    float2 p[kMaxQ1 + 1];       // p[t] = (w(t), w(t-1)); taps outside 0..Q-1 are zero
+};
+
 template <int Q>
-__device__ __forceinline__ void os_pass_1d_paired(const float *sx, float *so, const Taps1D &taps, int lane)
+__device__ __forceinline__ void os_pass_1d_paired(const float *sx, float *so, const Taps1D &taps,
+                                                  const Taps1DPairs &tp, int lane)
 {
     constexpr int M = R1 / 2;
     float X[R1];
@@ -133,7 +139,7 @@ __device__ __forceinline__ void os_pass_1d_paired(const float *sx, float *so, co
             } else if (t == Q) {
                 Z[m].y = fmaf(D[2 * m].x, taps.w[Q - 1], Z[m].y);
             } else {
-                Z[m] = __ffma2_rn(D[2 * m], make_float2(taps.w[t], taps.w[t - 1]), Z[m]);
+                Z[m] = __ffma2_rn(D[2 * m], tp.p[t], Z[m]);
             }
         }
         if (t < Q) {
@@ -183,6 +189,46 @@ __device__ __forceinline__ void is_pass_1d(const float *sx, float *so, const Tap
         const int off = lane * R1 + 4 * g - kShift;
         if (off >= 0 && off < kWarpOut1)
             *reinterpret_cast<float4 *>(so + off) = make_float4(Z[4 * g], Z[4 * g + 1], Z[4 * g + 2], Z[4 * g + 3]);
+    }
+}
+
+// ---- input-stationary, paired form for the longer filters (Q >= 12).  The sums of two neighbouring outputs
+// o (even) and o+1 travel TOGETHER in one 64-bit register pair: PE s adds x(s)*w(s-o) to the first and
+// x(s)*w(s-o-1) to the second, i.e. ONE packed fp32x2 FMA with the multiplicand (x(s), x(s)) and the aligned
+// tap pair (w(t), w(t-1)), t = s-o, from the kernel parameters.  The pair of outputs (o, o+1) sits in PE
+// o+t at step t, so the PEs with the parity of t hold the live pairs: Q+1 steps of R1/2 packed FMAs replace
+// Q steps of R1 scalar ones; the pairs move one PE up per step as before (lane-to-lane every second step).
+// The first and the last step touch only one sum of each pair and use scalar arithmetic, so that no input
+// outside an output's window enters its sum.
+template <int Q>
+__device__ __forceinline__ void is_pass_1d_paired(const float *sx, float *so, const Taps1D &taps,
+                                                  const Taps1DPairs &tp, int lane)
+{
+    float X[R1];
+    load_lane_block(sx + lane * R1, X);
+    float2 D[R1], P[R1];
+#pragma unroll
+    for (int j = 0; j < R1; ++j) D[j] = make_float2(X[j], X[j]);
+#pragma unroll
+    for (int j = 0; j < R1; j += 2) P[j] = make_float2(X[j] * taps.w[0], 0.f);
+#pragma unroll
+    for (int t = 1; t <= Q; ++t) {
+        float2 up = make_float2(0.f, 0.f);
+        if (t % 2 == 0)                                  // lane 0 keeps its own: invalid PEs
+            up = make_float2(__shfl_up_sync(kFullMask, P[R1 - 1].x, 1), __shfl_up_sync(kFullMask, P[R1 - 1].y, 1));
+#pragma unroll
+        for (int j = R1 - 1; j >= 0; --j) {
+            if (j % 2 != t % 2) continue;
+            const float2 prev = j == 0 ? up : P[j - 1];
+            if (t == Q) P[j] = make_float2(prev.x, fmaf(X[j], taps.w[Q - 1], prev.y));
+            else P[j] = __ffma2_rn(D[j], tp.p[t], prev);
+        }
+    }
+    // PE s (parity of Q) holds y(s-Q) and y(s-Q+1); the first PEs of the slice hold incomplete sums
+#pragma unroll
+    for (int j = Q % 2; j < R1; j += 2) {
+        const int off = lane * R1 + j - Q;
+        if (off >= 0 && off < kWarpOut1) *reinterpret_cast<float2 *>(so + off) = P[j];
     }
 }
 
@@ -356,7 +402,8 @@ __device__ __forceinline__ void fsm_pass_1d(const float *sx, float *so, const Ta
 
 template <int DESIGN, int Q, int WARPS, int K>
 __global__ void __launch_bounds__(Geo1D<DESIGN, WARPS>::kThreads)
-conv1d_f32_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, unsigned *status_word)
+conv1d_f32_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, const __grid_constant__ Taps1DPairs tpairs,
+                  unsigned *status_word)
 {
     using G = Geo1D<DESIGN, WARPS>;
     __shared__ __align__(128) float s_in[K][G::kTileIn];
@@ -415,8 +462,9 @@ conv1d_f32_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, unsig
 
             const float *sx = s_in[k] + warp * G::kWarpOut;
             float *so = s_out[k] + warp * G::kWarpOut;
-            if (DESIGN == SYSCONV_OS && Q >= 12) os_pass_1d_paired<Q>(sx, so, taps, lane);
+            if (DESIGN == SYSCONV_OS && Q >= 12) os_pass_1d_paired<Q>(sx, so, taps, tpairs, lane);
             else if (DESIGN == SYSCONV_OS) os_pass_1d<Q>(sx, so, taps, lane);
+            else if (DESIGN == SYSCONV_IS && Q >= 12) is_pass_1d_paired<Q>(sx, so, taps, tpairs, lane);
             else if (DESIGN == SYSCONV_IS) is_pass_1d<Q>(sx, so, taps, lane);
             else if (DESIGN == SYSCONV_WS) ws_pass_1d<Q>(sx, so, taps, lane);
             else if (DESIGN == SYSCONV_FSM) fsm_pass_1d<Q>(sx, so, taps, lane);
@@ -448,7 +496,10 @@ cudaError_t launch_conv1d_f32_q(const Conv1DArgs &a, const Taps1D &taps, unsigne
     const long long ctas = (a.n_out + per_cta - 1) / per_cta;
     if (ctas > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
     dim3 grid(static_cast<unsigned>(ctas), static_cast<unsigned>(a.batch < 65535 ? a.batch : 65535));
-    conv1d_f32_kernel<DESIGN, Q, WARPS, K><<<grid, G::kThreads, 0, s>>>(a, taps, status_word);
+    Taps1DPairs tp;
+    for (int t = 0; t <= kMaxQ1; ++t)
+        tp.p[t] = make_float2(t < kMaxQ1 ? taps.w[t] : 0.f, t > 0 ? taps.w[t - 1] : 0.f);
+    conv1d_f32_kernel<DESIGN, Q, WARPS, K><<<grid, G::kThreads, 0, s>>>(a, taps, tp, status_word);
     return cudaGetLastError();
 }
 
