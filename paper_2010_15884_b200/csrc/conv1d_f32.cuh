@@ -28,22 +28,22 @@
 namespace sysconv {
 
 // Tile geometry of a design.  OS and IS: each warp turns 640 inputs into 608 outputs.  WS: each warp
-// holds 16 two-lane arrays that stream 76 outputs each (1216 outputs per warp).  A tile is WARPS
+// holds 32 one-lane arrays that stream 76 outputs each (2432 outputs per warp).  A tile is WARPS
 // warp slices plus a 32-element halo (the halo budget is 32 whatever Q).
 template <int DESIGN, int WARPS>
 struct Geo1D {
     static constexpr int kWarps = WARPS;
-    static constexpr int kWarpOut = DESIGN == SYSCONV_WS ? kWsArrays1 * kWsSeg1 : kWarpOut1;
+    static constexpr int kWarpOut = DESIGN == SYSCONV_WS ? kLanes * kWsSeg1 : kWarpOut1;
     static constexpr int kThreads = kWarps * kLanes;
     static constexpr int kTileOut = kWarps * kWarpOut;     // outputs per CTA tile
     static constexpr int kTileIn = kTileOut + kHalo1;      // inputs per CTA tile
 };
 // shape used by the library (measured best on B200): two warps and two tiles per CTA; WS one warp per CTA
-// with one (twice as large) tile, two for the longer filters
+// with one (four times as large) tile
 template <int DESIGN, int Q>
 struct DefaultShape1D {
     static constexpr int kWarps = DESIGN == SYSCONV_WS ? 1 : 2;
-    static constexpr int kTiles = DESIGN == SYSCONV_WS ? (Q > 16 ? 2 : 1) : 2;
+    static constexpr int kTiles = DESIGN == SYSCONV_WS ? 1 : 2;
 };
 
 // ---- ordinary-load staging (ragged or unaligned tiles) ------------------------
@@ -232,75 +232,69 @@ __device__ __forceinline__ void is_pass_1d_paired(const float *sx, float *so, co
     }
 }
 
-// ---- weight-stationary (BSM, Table 2): PE s keeps w(s); at step t the input
-// x(t) is broadcast to the array, Z_s <- Z_{s-1} + x(t) * w(s), PE 0 starts a new
-// sum and the last PE emits y(t-(Q-1)).  An array has only Q PEs, so a warp holds
-// sixteen arrays of two lanes (RW PEs per lane, unused PEs keep a zero tap; the
-// array length QP = 2*RW is kept a multiple of four so that outputs leave as
-// aligned 128-bit words); array a streams the 76-output segment a of the warp's
-// 1216-output slice.  The broadcast is a same-address shared-memory read.
+// ---- weight-stationary (BSM, Table 2): PE s keeps w(s); at step t the input x(t) is broadcast to the
+// array, Z_s <- Z_{s-1} + x(t) * w(s), PE 0 starts a new sum and the last PE emits y(t-(Q-1)).
 //
-// Arrays neither fill nor drain separately: every array runs exactly the 76 steps
-// of its segment.  What array a+1 emits during its first QP-1 steps (sums over its
-// own inputs only) are the missing parts of the QP-1 sums still in flight in array a
-// when it stops, so they are stored into segment a's tail and array a adds its
-// registers to them afterwards.  Only the last array of the slice has no successor:
-// its tail gets the missing taps from a short direct sum over the slice's halo.
+// An array has only Q <= 32 PEs, so it is folded ENTIRELY into one lane (PE-to-PE transfer = register
+// renaming, no shuffle at all) and a warp holds 32 independent arrays; array a streams the 76-output
+// segment a of the warp's 2432-output slice (76 floats = 19 16-byte words: the lanes' 128-bit reads of
+// their segments fall in distinct banks).  All arrays hold the same filter, so the stationary weights
+// are uniform operands from the kernel parameters rather than a copy per lane.
+//
+// Paired form: the sums of two neighbouring outputs o (even) and o+1 travel together in one 64-bit
+// register pair; PE s adds x(t)*w(s) to the first and x(t)*w(s-1) to the second with ONE packed fp32x2
+// FMA (multiplicand (x(t), x(t)), multiplier the aligned tap pair (w(s), w(s-1))).  The pair (o, o+1)
+// sits in PE t-o at step t, so the PEs with the parity of t hold the live pairs: a step is Q/2 packed
+// FMAs.  PE 0 opens a pair with a scalar multiply, and the pair leaves PE Q-1 with its second sum one tap
+// short, which the emission adds with a scalar FMA: no zero tap ever multiplies an input.
+//
+// Arrays neither fill nor drain separately: every array runs exactly the 76 steps of its segment.  What
+// array a+1 emits during its first steps (sums over its own inputs only) are the missing parts of the
+// sums still in flight in array a when it stops, so they are stored into segment a's tail and array a
+// adds its registers to them afterwards.  Only the last array of the slice has no successor: its tail
+// gets the missing taps from a short direct sum over the slice's halo.
+constexpr int kWsSlice1 = kLanes * kWsSeg1;     // 2432 outputs per warp slice
+
 template <int Q>
-__device__ __forceinline__ void ws_pass_1d(const float *sx, float *so, const Taps1D &taps, int lane)
+__device__ __forceinline__ void ws_pass_1d(const float *sx, float *so, const Taps1D &taps, const Taps1DPairs &tp,
+                                           int lane)
 {
-    constexpr int RW = 2 * ((Q + 3) / 4);
-    constexpr int QP = RW * kWsLanes1;
     constexpr int kGroups = kWsSeg1 / 4;              // 76 time steps in groups of four
-    constexpr int kSlice = kWsArrays1 * kWsSeg1;      // 1216 outputs
-    static_assert(QP <= kHalo1 && QP <= kWsSeg1, "array longer than the halo or the segment");
-    const int m = lane & (kWsLanes1 - 1);
-    const int arr = lane / kWsLanes1;
-    float Wr[RW], Z[RW];
+    constexpr int kTail = Q - (Q % 2);                // outputs at the end of a segment still in flight
+    static_assert(Q <= kHalo1 && Q <= kWsSeg1, "array longer than the halo or the segment");
+    const float4 *xs4 = reinterpret_cast<const float4 *>(sx + lane * kWsSeg1);
+    float *yo = so + lane * kWsSeg1;
+    float2 P[Q];
 #pragma unroll
-    for (int i = 0; i < RW; ++i) {
-        const int s = m * RW + i;
-        Wr[i] = s < Q ? taps.w[s] : 0.f;
-        Z[i] = 0.f;
-    }
-    const float4 *xs4 = reinterpret_cast<const float4 *>(sx + arr * kWsSeg1);
-    float *yo = so + arr * kWsSeg1;
+    for (int s = 0; s < Q; ++s) P[s] = make_float2(0.f, 0.f);
 
-    // PEs beyond Q (they exist only on the pair's second lane, when Q is not a multiple of four) pass the
-    // partial sum on untouched: adding x(t) times their zero tap would let a non-finite input outside an
-    // output's window into its sum
-    const bool upper = m == kWsLanes1 - 1;
-    auto step = [&](float xb) -> float {
-        float up = __shfl_up_sync(kFullMask, Z[RW - 1], 1, kWsLanes1);
-        if (m == 0) up = 0.f;                          // PE 0: Z starts at zero
-#pragma unroll
-        for (int i = RW - 1; i > 0; --i) {
-            const float next = fmaf(xb, Wr[i], Z[i - 1]);
-            Z[i] = (RW + i >= Q && upper) ? Z[i - 1] : next;
-        }
-        Z[0] = (RW >= Q && upper) ? up : fmaf(xb, Wr[0], up);
-        return Z[RW - 1];                              // on the array's last lane: y(t-(QP-1))
-    };
-
-    float o0 = 0.f;
 #pragma unroll
     for (int k = 0; k < kGroups; ++k) {
         const float4 xv = xs4[k];                      // x(4k .. 4k+3) of this array's stream
-        const float o1 = step(xv.x);
-        const float o2 = step(xv.y);
-        const float o3 = step(xv.z);
-        // outputs 4k-QP .. 4k-QP+3 of this segment; negative positions are the tail of the previous
-        // segment and receive this array's share of those sums (the first array of the slice has no
-        // predecessor in the slice: the previous slice patches its own tail)
-        const int off = 4 * k - QP;
-        if (upper && (off >= 0 || arr > 0))
-            *reinterpret_cast<float4 *>(yo + off) = make_float4(o0, o1, o2, o3);
-        o0 = step(xv.w);
+        const float xr[4] = {xv.x, xv.y, xv.z, xv.w};
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int t = 4 * k + r;
+            const float x = xr[r];
+            if (t % 2 == Q % 2) {
+                // the pair that left PE Q-1 one step ago: outputs t-Q and t-Q+1 of this segment.  Negative
+                // positions are the tail of the previous segment and receive this array's share of those
+                // sums (the first array has no predecessor in the slice: the previous slice patches its own tail)
+                const float2 e = make_float2(P[Q - 1].x, fmaf(x, taps.w[Q - 1], P[Q - 1].y));
+                const int o = t - Q;
+                if (o >= 0 || lane > 0) *reinterpret_cast<float2 *>(yo + o) = e;
+            }
+            const float2 d = make_float2(x, x);
+#pragma unroll
+            for (int s = Q - 1; s >= 1; --s)
+                if (s % 2 == t % 2) P[s] = __ffma2_rn(d, tp.p[s], P[s - 1]);
+            if (t % 2 == 0) P[0] = make_float2(x * taps.w[0], 0.f);
+        }
     }
     // The last array's tail has no successor: store the taps it is missing, summed directly over the halo
-    // (output c = kSlice-1-j lacks the taps k > j); position kSlice-QP lacks nothing.
-    if (lane < QP) {
-        const int c = kSlice - 1 - lane;
+    // (output c = kWsSlice1-1-j lacks the taps k > j; the first position of an even-length tail lacks nothing).
+    if (lane < kTail) {
+        const int c = kWsSlice1 - 1 - lane;
         float acc = 0.f;
 #pragma unroll
         for (int k = 1; k < Q; ++k)
@@ -308,11 +302,11 @@ __device__ __forceinline__ void ws_pass_1d(const float *sx, float *so, const Tap
         so[c] = acc;
     }
     __syncwarp();
-    // PE s stopped while holding the sum of output 75-s of its segment (taps 0..s): add it to what is there
+    // the odd PEs stopped while holding the pairs of outputs 75-s and 76-s of the segment: add them to what is there
 #pragma unroll
-    for (int i = 0; i < RW; ++i) {
-        const int c = kWsSeg1 - 1 - (m * RW + i);
-        yo[c] += Z[i];
+    for (int s = 1; s < Q; s += 2) {
+        yo[kWsSeg1 - 1 - s] += P[s].x;
+        yo[kWsSeg1 - s] += P[s].y;
     }
 }
 
@@ -466,7 +460,7 @@ conv1d_f32_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, const
             else if (DESIGN == SYSCONV_OS) os_pass_1d<Q>(sx, so, taps, lane);
             else if (DESIGN == SYSCONV_IS && Q >= 12) is_pass_1d_paired<Q>(sx, so, taps, tpairs, lane);
             else if (DESIGN == SYSCONV_IS) is_pass_1d<Q>(sx, so, taps, lane);
-            else if (DESIGN == SYSCONV_WS) ws_pass_1d<Q>(sx, so, taps, lane);
+            else if (DESIGN == SYSCONV_WS) ws_pass_1d<Q>(sx, so, taps, tpairs, lane);
             else if (DESIGN == SYSCONV_FSM) fsm_pass_1d<Q>(sx, so, taps, lane);
             else if (DESIGN == SYSCONV_BFS) bfs_pass_1d<Q>(sx, so, taps, lane);
             else ffs_pass_1d<Q>(sx, so, taps, lane);
