@@ -470,15 +470,18 @@ def run_ours(args):
 
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch from the ncu captures summarised in
-# profiles/conv1d_f32_cfg2_kernels.md (full size) and profiles/conv2d_f32_cfg5_kernels.md (2 of 16 images,
-# scaled x8 here because traffic grows in proportion to the number of images).
+# profiles/conv1d_f32_cfg2_kernels.md (full size), profiles/conv2d_f32_cfg5_kernels.md (2 of 16 images, scaled x8
+# here because traffic grows in proportion to the number of images) and profiles/conv2d_u8_cfg4_kernels.md (full
+# size; the 33 MB of outputs stay dirty in L2 past the end of the kernel, so only the reads show).
 NCU_TRAFFIC = {
-    "cfg2 WS Q=4": 482353152, "cfg2 OS Q=4": 480993280, "cfg2 IS Q=4": 483138304,
-    "cfg2 WS Q=16": 487111424, "cfg2 OS Q=16": 485880064, "cfg2 IS Q=16": 483544320,
-    "cfg2 WS Q=32": 489855744, "cfg2 OS Q=32": 489574144, "cfg2 IS Q=32": 489446144,
-    "cfg5 WS 3x3": 8 * 239967488, "cfg5 OS 3x3": 8 * 226216960, "cfg5 IS 3x3": 8 * 224739072,
-    "cfg5 WS 9x9": 8 * 237750784, "cfg5 OS 9x9": 8 * 238917376, "cfg5 IS 9x9": 8 * 234722560,
-    "cfg5 WS 15x15": 8 * 238174976, "cfg5 OS 15x15": 8 * 241290752, "cfg5 IS 15x15": 8 * 241511424,
+    "cfg2 WS Q=4": 482644480, "cfg2 OS Q=4": 482553088, "cfg2 IS Q=4": 481613824,
+    "cfg2 WS Q=16": 481793280, "cfg2 OS Q=16": 482478848, "cfg2 IS Q=16": 482103296,
+    "cfg2 WS Q=32": 486940160, "cfg2 OS Q=32": 491869440, "cfg2 IS Q=32": 488185600,
+    "cfg5 WS 3x3": 8 * 240389376, "cfg5 OS 3x3": 8 * 224056064, "cfg5 IS 3x3": 8 * 225437184,
+    "cfg5 WS 9x9": 8 * 238213376, "cfg5 OS 9x9": 8 * 236435712, "cfg5 IS 9x9": 8 * 235231488,
+    "cfg5 WS 15x15": 8 * 238069760, "cfg5 OS 15x15": 8 * 240639232, "cfg5 IS 15x15": 8 * 240741888,
+    "cfg4 WS 3x3": 10990848, "cfg4 OS 3x3": 8317952, "cfg4 IS 3x3": 8303872,
+    "cfg4 WS 7x7": 10504192, "cfg4 OS 7x7": 8330240, "cfg4 IS 7x7": 8310016,
 }
 
 
