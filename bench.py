@@ -574,8 +574,24 @@ def six_designs_table(device, reps):
                 e0.record(); launch(); e1.record(); e1.synchronize()
                 ts.append(e0.elapsed_time(e1))
             times[name] = statistics.median(ts)
+        # the same six designs through the generic space-time executor (one PE per lane, CheckTime, run-time (P; s))
+        from paper_2010_15884_b200 import designspace
+        generic = {}
+        for name, (P, s) in designspace.PAPER_DESIGNS.items():
+            def launch_g(P=P, s=s, w=w, q=q, yd=yd):
+                st = B.sysconv1d_spacetime(xd.data_ptr(), n, w, q, yd.data_ptr(), P, s, stream)
+                if st != 0:
+                    raise B.SysconvError(st, "sysconv1d_spacetime")
+            launch_g()
+            ts = []
+            for _ in range(max(3, reps // 4)):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); launch_g(); e1.record(); e1.synchronize()
+                ts.append(e0.elapsed_time(e1))
+            generic[name] = statistics.median(ts)
         for name in enum:
             rows.append({"design": name, "filter": q, "ms": round(times[name], 5),
+                         "generic_executor_ms": round(generic[name], 4),
                          "gpix_s": round((n - q + 1) / (times[name] * 1e-3) / 1e9, 2),
                          "relative_to_FBS": round(times["FBS"] / times[name], 3),
                          "model_outturn_q5": model[name][0], "model_utilisation_pct_q5": model[name][1]})

@@ -134,6 +134,30 @@ int sysconv2d_strided(const void *x_dev, int width, int height, long long x_pitc
                       int dtype, int design, void *stream);
 
 /*
+ * Generic space-time-transform executor (Sections 2.1-2.2 and the generic code pattern of Section 4).
+ * The 1-D convolution UREs over the iteration space (c, q) are mapped by PE = p_c*c + p_q*q and
+ * time = s_c*c + s_q*q; the dependences, delays and PE distances are derived from (P, s) alone, so the six
+ * designs of Section 3.1 / Table 2 are (P; s) = SBM (1 1; 0 1), BSM (0 1; 1 1), FSM (0 1; 1 -1),
+ * BFS (1 0; 1 1), FFS (1 0; 2 1), FBS (1 0; 0 1), and any other valid transform runs too.  One PE per
+ * lane, register histories as deep as the delays, CheckTime on: a reference rendering, a small fraction of
+ * the speed of the folded kernels behind sysconv1d.
+ *
+ * sysconv_spacetime_describe (host only, no CUDA call): checks the validity conditions and reports
+ *   info[0..5]  PE distance and delay (in steps; 0 = broadcast) of the input, weight and partial-sum
+ *               dependences, info[6] outputs per array, info[7] PEs per array, info[8] time steps per array,
+ *               info[9] det(P; s);  name: the design letters (input B/F/S, weight B/F/S, sums M/S) + NUL.
+ *   info and name may be NULL.  Returns SYSCONV_EINVAL for a transform that breaks a validity condition
+ *   (P and s linearly dependent; sums that would accumulate within one time step) or q outside 1..32,
+ *   SYSCONV_EUNSUPPORTED for a valid one the executor does not cover (a delay above 4 steps, more than
+ *   32 PEs for one output).
+ * sysconv1d_spacetime: y_dev[c] = sum_k w_host[k] * x_dev[c+k], c < n-q+1, fp32, one signal, through that
+ *   array.  x_dev, y_dev DEVICE pointers, w_host HOST pointer; asynchronous on `stream`.
+ */
+int sysconv_spacetime_describe(int p_c, int p_q, int s_c, int s_q, int q, int *info, char *name);
+int sysconv1d_spacetime(const void *x_dev, long long n, const void *w_host, int q, void *y_dev,
+                        int p_c, int p_q, int s_c, int s_q, void *stream);
+
+/*
  * The same two operations for callers whose data lives in HOST memory
  * (densely packed: pitch = row length, batch stride = array size).  The call
  * enqueues the host-to-device copy of x into the caller's device workspace,

@@ -54,6 +54,10 @@ def load_library():
     lib.sysconv2d_strided.restype = _c_int
     lib.sysconv2d_strided.argtypes = [_vp, _c_int, _c_int, _c_ll, _c_ll, _vp, _c_int, _c_int, _c_int, _c_int, _vp,
                                       _c_ll, _c_ll, _c_int, _c_int, _c_int, _vp]
+    lib.sysconv_spacetime_describe.restype = _c_int
+    lib.sysconv_spacetime_describe.argtypes = [_c_int, _c_int, _c_int, _c_int, _c_int, _vp, _vp]
+    lib.sysconv1d_spacetime.restype = _c_int
+    lib.sysconv1d_spacetime.argtypes = [_vp, _c_ll, _vp, _c_int, _vp, _c_int, _c_int, _c_int, _c_int, _vp]
     lib.sysconv1d_host_workspace_bytes.restype = _c_ll
     lib.sysconv1d_host_workspace_bytes.argtypes = [_c_ll, _c_int, _c_int, _c_int]
     lib.sysconv2d_host_workspace_bytes.restype = _c_ll
@@ -153,6 +157,28 @@ def sysconv2d_strided(x_ptr, width, height, x_pitch, x_batch_stride, w_host, q, 
     return int(lib.sysconv2d_strided(_vp(x_ptr), width, height, x_pitch, x_batch_stride,
                                      w_host.ctypes.data_as(_vp), q, p, stride_c, stride_r, _vp(y_ptr), y_pitch,
                                      y_batch_stride, batch, dtype, design, _vp(stream_ptr)))
+
+
+def spacetime_describe(P, s, q):
+    """Plan of the generic executor for allocation row P = (p_c, p_q) and schedule row s = (s_c, s_q).
+
+    Returns (status, dict or None); the dict holds the design letters and, per dependence, PE distance and delay.
+    """
+    lib = load_library()
+    info = (ctypes.c_int * 10)()
+    name = ctypes.create_string_buffer(4)
+    st = int(lib.sysconv_spacetime_describe(int(P[0]), int(P[1]), int(s[0]), int(s[1]), int(q), info, name))
+    if st != 0:
+        return st, None
+    v = list(info)
+    return 0, {"name": name.value.decode(), "input": (v[0], v[1]), "weight": (v[2], v[3]), "sum": (v[4], v[5]),
+               "outputs_per_array": v[6], "pes": v[7], "steps": v[8], "det": v[9]}
+
+
+def sysconv1d_spacetime(x_ptr, n, w_host, q, y_ptr, P, s, stream_ptr):
+    lib = load_library()
+    return int(lib.sysconv1d_spacetime(_vp(x_ptr), n, w_host.ctypes.data_as(_vp), q, _vp(y_ptr), int(P[0]), int(P[1]),
+                                       int(s[0]), int(s[1]), _vp(stream_ptr)))
 
 
 def host_workspace_bytes(shape, filt, dtype=F32):

@@ -238,6 +238,32 @@ int sysconv2d_strided(const void *x_dev, int width, int height, long long x_pitc
     return finish(err, launches);
 }
 
+int sysconv_spacetime_describe(int p_c, int p_q, int s_c, int s_q, int q, int *info, char *name)
+{
+    return sysconv::spacetime_describe(p_c, p_q, s_c, s_q, q, info, name);
+}
+
+int sysconv1d_spacetime(const void *x_dev, long long n, const void *w_host, int q, void *y_dev, int p_c, int p_q, int s_c,
+                        int s_q, void *stream)
+{
+    using namespace sysconv;
+    if (!x_dev || !y_dev || !w_host) return SYSCONV_EINVAL;
+    if (q < 1 || n < q) return SYSCONV_EINVAL;
+    const long long n_out = n - q + 1;
+    if (overlaps(x_dev, (unsigned long long)n * 4ull, y_dev, (unsigned long long)n_out * 4ull)) return SYSCONV_EINVAL;
+    if (q > kMaxQ1) return SYSCONV_EUNSUPPORTED;
+    const int plan = spacetime_describe(p_c, p_q, s_c, s_q, q, nullptr, nullptr);
+    if (plan != SYSCONV_OK) return plan;
+    const DeviceInfo *d = device_info();
+    if (!d) return SYSCONV_ECUDA;
+    int status = SYSCONV_OK, launches = 0;
+    const cudaError_t err = launch_spacetime_conv1d(static_cast<const float *>(x_dev), n, static_cast<const float *>(w_host),
+                                                    q, static_cast<float *>(y_dev), p_c, p_q, s_c, s_q, d->sm_count,
+                                                    static_cast<cudaStream_t>(stream), &status, &launches);
+    if (status != SYSCONV_OK) return status;
+    return finish(err, launches);
+}
+
 int sysconv2d(const void *x_dev, int width, int height, long long x_pitch, long long x_batch_stride,
               const void *w_host, int q, int p, void *y_dev, long long y_pitch, long long y_batch_stride,
               int batch, int dtype, int design, void *stream)

@@ -25,7 +25,8 @@ def _declared_functions():
 
 def test_header_declares_the_expected_entry_points():
     names = _declared_functions()
-    for must in ("sysconv1d", "sysconv2d", "sysconv1d_strided", "sysconv2d_strided", "sysconv1d_host", "sysconv2d_host", "sysconv_status_string",
+    for must in ("sysconv1d", "sysconv2d", "sysconv1d_strided", "sysconv2d_strided", "sysconv_spacetime_describe",
+                 "sysconv1d_spacetime", "sysconv1d_host", "sysconv2d_host", "sysconv_status_string",
                  "sysconv_design_name", "sysconv_version", "sysconv_launch_count"):
         assert must in names
 

@@ -530,6 +530,75 @@ def test_2d_stride2_full_hd_sampled(cuda_device):
         assert_close_f32(y.cpu().numpy()[0][rows, cols], y_ref, s_ref, "sampled, %s" % B.DESIGN_NAMES[design])
 
 
+# ------------------------------------------------------------------------ generic space-time executor
+
+ST_PAPER = {"SBM": ((1, 1), (0, 1)), "BSM": ((0, 1), (1, 1)), "FSM": ((0, 1), (1, -1)), "BFS": ((1, 0), (1, 1)),
+            "FFS": ((1, 0), (2, 1)), "FBS": ((1, 0), (0, 1))}
+# other valid transforms: mirrored arrays, slower schedules, skewed allocations, a non-unimodular one
+ST_OTHER = [((-1, 0), (0, 1)), ((1, 0), (0, -1)), ((1, 0), (1, 2)), ((1, 0), (3, 1)), ((0, 1), (2, 1)),
+            ((1, 1), (1, -1)), ((1, -1), (0, 1)), ((1, 1), (-1, 2)), ((2, 1), (0, 1)), ((1, 2), (1, 1)),
+            ((0, -1), (1, 1)), ((1, 0), (-1, 1)), ((1, 1), (0, 2)), ((2, 0), (1, 1))]
+
+
+def run_spacetime(x, w, P, s, device):
+    n, q = x.shape[0], w.shape[0]
+    xd = torch.from_numpy(x).to(device)
+    yd = torch.full((n - q + 1 + 16,), CANARY, dtype=torch.float32, device=device)
+    st = B.sysconv1d_spacetime(xd.data_ptr(), n, w, q, yd.data_ptr(), P, s, torch.cuda.current_stream().cuda_stream)
+    assert st == 0, (P, s, B.status_string(st))
+    torch.cuda.synchronize()
+    yh = yd.cpu().numpy()
+    assert (yh[n - q + 1:] == CANARY).all()
+    return yh[:n - q + 1]
+
+
+@pytest.mark.parametrize("name", list(ST_PAPER))
+@pytest.mark.parametrize("q", [1, 2, 5, 8, 16, 31, 32])
+def test_spacetime_executor_runs_the_six_designs(cuda_device, name, q):
+    P, s = ST_PAPER[name]
+    x, ws = inputs.gen_1d_f32(5000 + q, [q], seed=700 + q)
+    y = run_spacetime(x, ws[q], P, s, cuda_device)
+    y_ref, s_ref = oracle.conv1d_f32(x, ws[q])
+    assert_close_f32(y, y_ref, s_ref, "%s q=%d" % (name, q))
+    st, info = B.spacetime_describe(P, s, q)
+    assert st == 0 and info["name"] == name
+
+
+@pytest.mark.parametrize("Ps", ST_OTHER, ids=lambda t: "P%d,%d_s%d,%d" % (t[0] + t[1]))
+def test_spacetime_executor_runs_other_valid_transforms(cuda_device, Ps):
+    P, s = Ps
+    for q, n in [(5, 777), (12, 4099), (1, 40), (3, 3)]:
+        st, info = B.spacetime_describe(P, s, q)
+        if st == 2:
+            continue                      # valid but not covered at this filter length (array too long)
+        assert st == 0
+        x, ws = inputs.gen_1d_f32(n, [q], seed=800 + q)
+        y = run_spacetime(x, ws[q], P, s, cuda_device)
+        y_ref, s_ref = oracle.conv1d_f32(x, ws[q])
+        assert_close_f32(y, y_ref, s_ref, "%s q=%d" % (Ps, q))
+
+
+def test_spacetime_executor_matches_the_folded_kernels_on_integers(cuda_device):
+    # integer-valued data: every order of summation is exact, so all designs must agree bit for bit
+    rng = np.random.default_rng(8)
+    x = rng.integers(-8, 9, 20000).astype(np.float32)
+    w = rng.integers(-4, 5, 7).astype(np.float32)
+    ref = B.conv1d(torch.from_numpy(x).to(cuda_device), w, B.OS).cpu().numpy()
+    for P, s in list(ST_PAPER.values()) + ST_OTHER[:6]:
+        np.testing.assert_array_equal(run_spacetime(x, w, P, s, cuda_device), ref)
+
+
+def test_spacetime_executor_rejects_invalid_transforms(cuda_device):
+    x = torch.zeros(100, device=cuda_device)
+    y = torch.zeros(96, device=cuda_device)
+    w = np.ones(5, np.float32)
+    s0 = torch.cuda.current_stream().cuda_stream
+    assert B.sysconv1d_spacetime(x.data_ptr(), 100, w, 5, y.data_ptr(), (1, 1), (1, 1), s0) == 1
+    assert B.sysconv1d_spacetime(x.data_ptr(), 100, w, 5, y.data_ptr(), (0, 1), (1, 0), s0) == 1
+    assert B.sysconv1d_spacetime(x.data_ptr(), 100, w, 5, y.data_ptr(), (1, 0), (5, 1), s0) == 2
+    assert B.sysconv1d_spacetime(x.data_ptr(), 100, w, 5, x.data_ptr(), (1, 0), (0, 1), s0) == 1     # x and y overlap
+
+
 # ------------------------------------------------------------------------ integer
 
 
