@@ -49,8 +49,10 @@
  *     would multiply them by the non-finite value: the 2-D output-stationary
  *     kernels with 12 or more filter rows (the output rows directly above and
  *     below the affected rows may turn NaN) and the 2-D weight-stationary
- *     kernels when q is not a multiple of 4 (up to three outputs to the left
- *     of the affected columns may turn NaN).  Finite data is unaffected.
+ *     kernel used for small problems (fewer than 592 blocks of 128 output rows
+ *     x 128 output columns over all images) when q is not a multiple of 4 (up
+ *     to three outputs to the left of the affected columns may turn NaN).
+ *     Finite data is unaffected.
  *   - Errors: every function returns a sysconv_status; nothing throws, aborts
  *     or traps.  SYSCONV_EINVAL: null pointer, non-positive size, filter larger
  *     than the input, pitch/stride smaller than the row/array, unknown enum.

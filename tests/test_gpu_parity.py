@@ -390,6 +390,37 @@ def test_2d_non_finite_inputs_stay_inside_their_windows(cuda_device, design, pq)
     assert (np.abs(y[loose] - y_ref[loose]) <= TOL * s_ref[loose]).all()
 
 
+# The fp32 weight-stationary 2-D kernel with one array per lane runs when the problem gives its one-warp CTAs
+# enough work (bands of 128 rows x segments of >= 128 columns x images >= 592); these cases are sized for it.
+WS_LANE_BATCH = 150
+
+
+@pytest.mark.parametrize("pq", [(1, 1), (3, 3), (5, 5), (2, 11), (13, 4), (9, 9), (15, 15), (7, 10), (15, 1), (1, 15),
+                                (4, 9), (6, 2)], ids=lambda f: "%dx%d" % f)
+def test_2d_ws_one_array_per_lane_kernel(cuda_device, pq):
+    p, q = pq
+    x, ws = inputs.gen_2d_f32(261, 150, [pq], seed=900 + 16 * p + q, batch=WS_LANE_BATCH)
+    assert ((150 - p + 1 + 127) // 128) * ((261 - q + 1 + 127) // 128) * WS_LANE_BATCH >= 592
+    check_2d(x, ws[pq], B.WS, cuda_device)
+
+
+def test_2d_ws_one_array_per_lane_kernel_layouts_and_non_finite(cuda_device):
+    pq = (5, 7)
+    x, ws = inputs.gen_2d_f32(300, 150, [pq], seed=77, batch=WS_LANE_BATCH)
+    assert ((150 - 5 + 1 + 127) // 128) * ((300 - 7 + 1 + 127) // 128) * WS_LANE_BATCH >= 592
+    check_2d(x, ws[pq], B.WS, cuda_device, x_pitch=307, y_pitch=299, x_off=1, y_off=3)
+    check_2d(x, ws[pq], B.WS, cuda_device, x_pitch=304, y_pitch=296, x_off=4, y_off=4)
+    # this kernel applies no zero taps: a non-finite pixel must affect exactly the outputs whose window holds it
+    for r, c, v in BAD_PIXELS:
+        x[3, r, c] = v
+    with np.errstate(invalid="ignore"):
+        y_ref, s_ref = oracle.conv2d_f32(x[3], ws[pq])
+    y = run_2d(x, ws[pq], B.WS, cuda_device)[3].astype(np.float64)
+    fin = np.isfinite(y_ref)
+    assert (np.isfinite(y) == fin).all()
+    assert (np.abs(y[fin] - y_ref[fin]) <= TOL * s_ref[fin]).all()
+
+
 # ------------------------------------------------------------------------ stride 2 (Table 2, cell 6)
 
 STRIDED_DESIGNS = [B.OS, B.IS]
