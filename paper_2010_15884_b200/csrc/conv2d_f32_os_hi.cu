@@ -1,0 +1,11 @@
+// 2-D fp32 kernels of the output-stationary (FBS) design, filter heights 11..15 (all widths 1..15).
+#include "conv2d_kernels.cuh"
+
+namespace sysconv {
+
+cudaError_t launch_conv2d_f32_os_hi(const Conv2DArgs &a, const float *w, int q, int p, cudaStream_t s, int *launches)
+{
+    return launch_conv2d_range<F32Traits, SYSCONV_OS, 11, kMaxP2>(a, w, q, p, s, launches);
+}
+
+}  // namespace sysconv

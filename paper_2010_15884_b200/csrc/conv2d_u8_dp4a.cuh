@@ -183,4 +183,15 @@ cudaError_t launch_conv2d_u8_os_dp4a(const Conv2DArgs &a, const Taps2DInt &t, cu
     return cudaGetLastError();
 }
 
+// uint8 rows that start 4-byte aligned run on the packed (dp4a) kernel
+template <int P, int Q>
+struct FastPath2D<U8Traits, SYSCONV_OS, P, Q> {
+    static bool launch(const Conv2DArgs &a, const Taps2DInt &taps, cudaStream_t s, cudaError_t *err)
+    {
+        if (!u8_dp4a_eligible(a)) return false;
+        *err = launch_conv2d_u8_os_dp4a<P, Q>(a, taps, s);
+        return true;
+    }
+};
+
 }  // namespace sysconv
