@@ -276,8 +276,9 @@ def detail_rows(cases, hbm_gbs, peak_kind, sm_max):
 def oracle_sample(cfg_id):
     """Time the oracle, as it stands, on a bounded sample of the configuration.
 
-    Returns (outputs, seconds, threads, description).  1-D: one pass per filter length over the first
-    2^24 samples.  2-D: one pass per filter size over the first 1024 rows of image 0.
+    Returns (outputs, seconds, threads, description).  1-D: passes per filter length over the first
+    2^24 samples.  2-D: passes per filter size over the first 1024 rows of image 0.  The passes repeat until
+    about one second of wall time (10-20 core-seconds on this machine's host cores) has gone by.
     """
     import oracle
     from paper_2010_15884_b200 import inputs
@@ -287,18 +288,22 @@ def oracle_sample(cfg_id):
     if kind == "1d_f32":
         x = x[: 1 << 24]
         oracle.conv1d_f32(x[: 1 << 16], next(iter(ws.values())), want_scale=False)   # load + warm
-        t0 = time.perf_counter()
-        for w in ws.values():
-            outs += oracle.conv1d_f32(x, w, want_scale=False)[0].size
-        what = "one fp64 pass of Eq. 2 per filter length over the first %d samples" % x.shape[0]
+        t0, reps = time.perf_counter(), 0
+        while reps < 50 and time.perf_counter() - t0 < 1.0:
+            for w in ws.values():
+                outs += oracle.conv1d_f32(x, w, want_scale=False)[0].size
+            reps += 1
+        what = "%d fp64 passes of Eq. 2 per filter length over the first %d samples" % (reps, x.shape[0])
     else:
         img = np.ascontiguousarray(x[0][:1024])
         f = oracle.conv2d_f32 if kind == "2d_f32" else (lambda a, b, want_scale=False: (oracle.conv2d_u8s8_s32(a, b), None))
         f(img[:32], next(iter(ws.values())), want_scale=False)
-        t0 = time.perf_counter()
-        for w in ws.values():
-            outs += f(img, w, want_scale=False)[0].size
-        what = "one pass of Eq. 3 per filter size over the first %d rows of image 0" % img.shape[0]
+        t0, reps = time.perf_counter(), 0
+        while reps < 50 and time.perf_counter() - t0 < 1.0:
+            for w in ws.values():
+                outs += f(img, w, want_scale=False)[0].size
+            reps += 1
+        what = "%d passes of Eq. 3 per filter size over the first %d rows of image 0" % (reps, img.shape[0])
     return outs, time.perf_counter() - t0, oracle.num_threads(), what
 
 
@@ -456,7 +461,7 @@ def run_ours(args):
             outs, secs, cores, what = oracle_sample(cfg_id)
             line["cpu_baseline"] = {
                 "value": round(outs / secs / 1e9, 4), "unit": "Gpix/s", "cores": cores, "kind": "oracle",
-                "sample": "%s of configuration %d (%.1f s)" % (what, cfg_id, secs)}
+                "sample": "%s of configuration %d (%.1f s wall on %d threads)" % (what, cfg_id, secs, cores)}
         line["per_kernel"] = detail_rows(cases, hbm_gbs, peak_kind, sm_max)
         if not args.no_detail and world == 1:
             del cases, keep
@@ -608,7 +613,25 @@ def all_config_detail(device, hbm_gbs, peak_kind, sm_max, skip, reps):
         cases, keep = build_cases(cfg_id, device)
         small = max(c.alg_bytes for c in cases) < 256e6
         time_cases_individually(cases, 3, reps, flush if small else None)
-        rows += detail_rows(cases, hbm_gbs, peak_kind, sm_max)
+        new_rows = detail_rows(cases, hbm_gbs, peak_kind, sm_max)
+        if small:
+            # yardstick for the launch/latency-bound sizes: a plain device-to-device copy that moves the same
+            # number of bytes (half read, half written), timed the same way (L2 flushed before every launch)
+            for c, row in zip(cases, new_rows):
+                half = max(int(c.alg_bytes) // 8 * 4, 4)
+                src = torch.empty(half, dtype=torch.uint8, device=device)
+                dst = torch.empty(half, dtype=torch.uint8, device=device)
+                ts = []
+                for i in range(3 + reps):
+                    flush.add_(1.0)
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record(); dst.copy_(src); e1.record(); e1.synchronize()
+                    if i >= 3:
+                        ts.append(e0.elapsed_time(e1))
+                row["copy_same_bytes_ms"] = round(statistics.median(ts), 5)
+                row["frac_of_copy"] = round(statistics.median(ts) / row["ms_median"], 3)
+                del src, dst
+        rows += new_rows
         del cases, keep
         torch.cuda.empty_cache()
     cases, keep = build_strided_cases(device)
