@@ -469,6 +469,7 @@ def run_ours(args):
             line["detail"] = all_config_detail(device, hbm_gbs, peak_kind, sm_max, skip=cfg_id,
                                                reps=args.detail_reps)
             line["six_designs_n2p24"] = six_designs_table(device, args.detail_reps)
+            line["cfg1_step_in_cuda_graph"] = graph_replay_ms(1, device, 200)
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -547,6 +548,38 @@ def run_e2e(cfg_id, device, args, world):
             "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": steps,
             "ms_per_step": round(ms / steps, 3),
             "path": "sysconv1d_host/sysconv2d_host: pinned host -> device workspace -> kernel -> pinned host"}
+
+
+def graph_replay_ms(cfg_id, device, reps):
+    """One step of a launch-bound configuration (every filter x design) captured once in a CUDA graph and replayed:
+    ms per step by replay and by direct launches (CUDA events around `reps` back-to-back steps, no L2 flush)."""
+    import torch
+    cases, keep = build_cases(cfg_id, device)
+    for c in cases:
+        c.launch()                       # first-call set-up happens outside the capture
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        cases_s, keep_s = build_cases(cfg_id, device)      # launch closures bound to the side stream
+        torch.cuda.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            for c in cases_s:
+                c.launch()
+    out = {}
+    for name, run in (("graph_replay", graph.replay), ("direct_launches", lambda: [c.launch() for c in cases])):
+        for _ in range(3):
+            run()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            run()
+        e1.record(); e1.synchronize()
+        out[name + "_ms_per_step"] = round(e0.elapsed_time(e1) / reps, 5)
+    out["launches_per_step"] = len(cases)
+    del cases, keep, cases_s, keep_s
+    return out
 
 
 def six_designs_table(device, reps):

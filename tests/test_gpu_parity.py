@@ -630,6 +630,36 @@ def test_spacetime_executor_rejects_invalid_transforms(cuda_device):
     assert B.sysconv1d_spacetime(x.data_ptr(), 100, w, 5, x.data_ptr(), (1, 0), (0, 1), s0) == 1     # x and y overlap
 
 
+# ------------------------------------------------------------------------ launches inside a CUDA graph
+
+
+def test_device_entry_points_replay_inside_a_cuda_graph(cuda_device):
+    """The device-pointer entry points only enqueue kernels on the caller's stream, so a launch-bound loop of
+    small problems can be captured once and replayed; the replayed results must equal the direct ones."""
+    x1, ws1 = inputs.make_config(1)
+    x2, ws2 = inputs.gen_2d_f32(200, 90, [(3, 3)], seed=5)
+    xd1, xd2 = torch.from_numpy(x1).to(cuda_device), torch.from_numpy(x2).to(cuda_device)
+    w1, w2 = ws1[8], ws2[(3, 3)]
+    direct = [B.conv1d(xd1, w1, d) for d in DESIGNS] + [B.conv2d(xd2, w2, d) for d in DESIGNS]   # also first-call set-up
+    outs = [torch.zeros_like(t) for t in direct]
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for i, d in enumerate(DESIGNS):
+                B.conv1d(xd1, w1, d, out=outs[i], stream=side)
+                B.conv2d(xd2, w2, d, out=outs[3 + i], stream=side)
+    for o in outs:
+        o.zero_()
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    for got, want in zip(outs, direct):
+        assert torch.equal(got, want)
+    assert B.device_status() == 0
+
+
 # ------------------------------------------------------------------------ integer
 
 
