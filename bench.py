@@ -480,14 +480,14 @@ def run_ours(args):
 # here because traffic grows in proportion to the number of images) and profiles/conv2d_u8_cfg4_kernels.md (full
 # size; the 33 MB of outputs stay dirty in L2 past the end of the kernel, so only the reads show).
 NCU_TRAFFIC = {
-    "cfg2 WS Q=4": 482644480, "cfg2 OS Q=4": 482553088, "cfg2 IS Q=4": 481613824,
-    "cfg2 WS Q=16": 481793280, "cfg2 OS Q=16": 482478848, "cfg2 IS Q=16": 482103296,
-    "cfg2 WS Q=32": 486940160, "cfg2 OS Q=32": 491869440, "cfg2 IS Q=32": 488185600,
-    "cfg5 WS 3x3": 8 * 240389376, "cfg5 OS 3x3": 8 * 224056064, "cfg5 IS 3x3": 8 * 225437184,
-    "cfg5 WS 9x9": 8 * 238213376, "cfg5 OS 9x9": 8 * 236435712, "cfg5 IS 9x9": 8 * 235231488,
-    "cfg5 WS 15x15": 8 * 238069760, "cfg5 OS 15x15": 8 * 240639232, "cfg5 IS 15x15": 8 * 240741888,
-    "cfg4 WS 3x3": 10990848, "cfg4 OS 3x3": 8317952, "cfg4 IS 3x3": 8303872,
-    "cfg4 WS 7x7": 10504192, "cfg4 OS 7x7": 8330240, "cfg4 IS 7x7": 8310016,
+    "cfg2 WS Q=4": 482735616, "cfg2 OS Q=4": 483311616, "cfg2 IS Q=4": 482604800,
+    "cfg2 WS Q=16": 482735616, "cfg2 OS Q=16": 484164608, "cfg2 IS Q=16": 482969856,
+    "cfg2 WS Q=32": 486377472, "cfg2 OS Q=32": 487852032, "cfg2 IS Q=32": 486862848,
+    "cfg5 WS 3x3": 8 * 281386752, "cfg5 OS 3x3": 8 * 223146240, "cfg5 IS 3x3": 8 * 225374976,
+    "cfg5 WS 9x9": 8 * 270929664, "cfg5 OS 9x9": 8 * 235896832, "cfg5 IS 9x9": 8 * 235905280,
+    "cfg5 WS 15x15": 8 * 282466816, "cfg5 OS 15x15": 8 * 238883840, "cfg5 IS 15x15": 8 * 240188928,
+    "cfg4 WS 3x3": 10941184, "cfg4 OS 3x3": 8308224, "cfg4 IS 3x3": 8303872,
+    "cfg4 WS 7x7": 10521856, "cfg4 OS 7x7": 8306944, "cfg4 IS 7x7": 8310272,
 }
 
 
