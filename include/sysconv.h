@@ -192,6 +192,21 @@ int sysconv2d_host(const void *x_host, int width, int height, const void *w_host
                    void *workspace_dev, long long workspace_bytes, void *stream);
 
 /*
+ * Several filters / designs over ONE host signal in one call (the shape of an experiment of the paper: the same
+ * input through every design and filter size).  The signal crosses to the device once; job j convolves it with
+ * the q[j] taps at w_host[j] by design[j] and its n-q[j]+1 outputs go to y_host[j].  Chunked like
+ * sysconv1d_host: the copy in of chunk c+1, the kernels of chunk c and the copies out of chunk c-1 overlap.
+ *   count                  1 .. 64 jobs;  w_host, y_host: HOST arrays of `count` HOST pointers;  q, design: HOST
+ *                          arrays of `count` ints
+ *   workspace_dev / bytes  at least sysconv1d_host_multi_workspace_bytes(n, q, count, dtype), 256-byte aligned
+ * The y_host[j] must not overlap each other or x_host.  fp32 only (SYSCONV_EUNSUPPORTED otherwise).
+ */
+long long sysconv1d_host_multi_workspace_bytes(long long n, const int *q, int count, int dtype);
+int sysconv1d_host_multi(const void *x_host, long long n, int count,
+                         const void *const *w_host, const int *q, const int *design, void *const *y_host,
+                         int dtype, void *workspace_dev, long long workspace_bytes, void *stream);
+
+/*
  * sysconv1d_host for callers that cannot allocate device memory.  (The paper has
  * no counterpart: this is a packaging variant, not a systolic design.)
  *

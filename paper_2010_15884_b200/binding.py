@@ -67,6 +67,10 @@ def load_library():
     lib.sysconv2d_host.restype = _c_int
     lib.sysconv2d_host.argtypes = [_vp, _c_int, _c_int, _vp, _c_int, _c_int, _vp, _c_int, _c_int, _c_int,
                                    _vp, _c_ll, _vp]
+    lib.sysconv1d_host_multi_workspace_bytes.restype = _c_ll
+    lib.sysconv1d_host_multi_workspace_bytes.argtypes = [_c_ll, _vp, _c_int, _c_int]
+    lib.sysconv1d_host_multi.restype = _c_int
+    lib.sysconv1d_host_multi.argtypes = [_vp, _c_ll, _c_int, _vp, _vp, _vp, _vp, _c_int, _vp, _c_ll, _vp]
     lib.sysconv1d_host_static.restype = _c_int
     lib.sysconv1d_host_static.argtypes = [_vp, _c_ll, _vp, _c_int, _vp, _c_int, _c_int, _c_int, _vp]
     lib.sysconv_static_scratch_bytes.restype = _c_ll
@@ -202,6 +206,31 @@ def sysconv1d_host(x_host, w_host, y_host, design, workspace, stream=None, dtype
                             _vp(_stream_ptr(stream)))
     if st != 0:
         raise SysconvError(st, "sysconv1d_host")
+
+
+def host_multi_workspace_bytes(n, qs, dtype=F32):
+    lib = load_library()
+    arr = (ctypes.c_int * len(qs))(*[int(v) for v in qs])
+    return int(lib.sysconv1d_host_multi_workspace_bytes(int(n), arr, len(qs), dtype))
+
+
+def sysconv1d_host_multi(x_host, jobs, workspace, stream=None, dtype=F32):
+    """One host signal through several (taps, design, y_host) jobs; the signal is copied to the device once.
+
+    jobs: sequence of (w_host, design, y_host); x_host and the y_host are host arrays/tensors (pinned for overlap).
+    """
+    lib = load_library()
+    n = int(tuple(x_host.shape)[0])
+    taps = [_host_taps(w, dtype, 1) for w, _, _ in jobs]
+    count = len(jobs)
+    w_ptrs = (ctypes.c_void_p * count)(*[t.ctypes.data for t in taps])
+    y_ptrs = (ctypes.c_void_p * count)(*[_data_ptr(y) for _, _, y in jobs])
+    qs = (ctypes.c_int * count)(*[int(t.shape[0]) for t in taps])
+    ds = (ctypes.c_int * count)(*[_design(d) for _, d, _ in jobs])
+    st = lib.sysconv1d_host_multi(_vp(_data_ptr(x_host)), n, count, w_ptrs, qs, ds, y_ptrs, dtype,
+                                  _vp(workspace.data_ptr()), workspace.numel(), _vp(_stream_ptr(stream)))
+    if st != 0:
+        raise SysconvError(st, "sysconv1d_host_multi")
 
 
 def static_scratch_bytes():

@@ -373,6 +373,86 @@ int sysconv1d_host(const void *x_host, long long n, const void *w_host, int q, v
     return pipe->join(s) ? SYSCONV_OK : SYSCONV_ECUDA;
 }
 
+long long sysconv1d_host_multi_workspace_bytes(long long n, const int *q, int count, int dtype)
+{
+    if (!q || count < 1 || count > 64 || dtype != SYSCONV_F32) return -1;
+    long long total = align256(n * 4LL);
+    for (int j = 0; j < count; ++j) {
+        if (q[j] < 1 || n < q[j]) return -1;
+        total += align256((n - q[j] + 1) * 4LL);
+    }
+    return total;
+}
+
+int sysconv1d_host_multi(const void *x_host, long long n, int count, const void *const *w_host, const int *q,
+                         const int *design, void *const *y_host, int dtype, void *workspace_dev,
+                         long long workspace_bytes, void *stream)
+{
+    if (!x_host || !w_host || !q || !design || !y_host || !workspace_dev) return SYSCONV_EINVAL;
+    if (count < 1 || count > 64) return SYSCONV_EINVAL;
+    if (dtype != SYSCONV_F32 && dtype != SYSCONV_U8S8_S32) return SYSCONV_EINVAL;
+    if (dtype != SYSCONV_F32) return SYSCONV_EUNSUPPORTED;
+    for (int j = 0; j < count; ++j) {
+        if (!w_host[j] || !y_host[j] || q[j] < 1 || n < q[j] || !valid_enums(dtype, design[j])) return SYSCONV_EINVAL;
+        if (q[j] > sysconv::kMaxQ1) return SYSCONV_EUNSUPPORTED;
+    }
+    const long long need = sysconv1d_host_multi_workspace_bytes(n, q, count, dtype);
+    if (need < 0 || workspace_bytes < need) return SYSCONV_EINVAL;
+    if ((reinterpret_cast<unsigned long long>(workspace_dev) & 255ull) != 0) return SYSCONV_EINVAL;
+    int q_min = q[0], q_max = q[0];
+    for (int j = 1; j < count; ++j) { q_min = q[j] < q_min ? q[j] : q_min; q_max = q[j] > q_max ? q[j] : q_max; }
+    char *xd = static_cast<char *>(workspace_dev);
+    char *yd[64];
+    {
+        char *at = xd + align256(n * 4LL);
+        for (int j = 0; j < count; ++j) { yd[j] = at; at += align256((n - q[j] + 1) * 4LL); }
+    }
+    HostPipe *pipe = host_pipe();
+    if (!pipe) return SYSCONV_ECUDA;
+    std::lock_guard<std::mutex> lock(pipe->busy);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // chunks of output positions, the same for every job (a job's last chunk ends at its own n - q + 1)
+    const long long span = n - q_min + 1;
+    long long chunks = span / (1LL << 20);
+    if (chunks > kMaxPipeChunks) chunks = kMaxPipeChunks;
+    if (chunks < 1) chunks = 1;
+    long long len = (span + chunks - 1) / chunks;
+    len = (len + 9727) / 9728 * 9728;                    // whole tiles of every design; keeps 16-byte alignment
+    if (!pipe->fork(s)) return SYSCONV_ECUDA;
+    int c = 0;
+    long long copied = 0;                                // inputs [0, copied) are on the device
+    for (long long o0 = 0; o0 < span; o0 += len, ++c) {
+        const long long o1 = o0 + len < span ? o0 + len : span;
+        long long in1 = o1 + q_max - 1;
+        if (in1 > n) in1 = n;
+        if (in1 > copied) {
+            if (cudaMemcpyAsync(xd + copied * 4, static_cast<const char *>(x_host) + copied * 4, (in1 - copied) * 4,
+                                cudaMemcpyHostToDevice, pipe->h2d) != cudaSuccess) return SYSCONV_ECUDA;
+            copied = in1;
+        }
+        if (cudaEventRecord(pipe->in_done[c], pipe->h2d) != cudaSuccess) return SYSCONV_ECUDA;
+        if (cudaStreamWaitEvent(s, pipe->in_done[c], 0) != cudaSuccess) return SYSCONV_ECUDA;
+        for (int j = 0; j < count; ++j) {
+            const long long n_out = n - q[j] + 1;
+            const long long e1 = o1 < n_out ? o1 : n_out;
+            if (o0 >= e1) continue;
+            const int st = sysconv1d(xd + o0 * 4, (e1 - o0) + q[j] - 1, 0, w_host[j], q[j], yd[j] + o0 * 4, 0, 1, dtype,
+                                     design[j], stream);
+            if (st != SYSCONV_OK) { pipe->join(s); return st; }
+        }
+        if (cudaEventRecord(pipe->k_done[c], s) != cudaSuccess) return SYSCONV_ECUDA;
+        if (cudaStreamWaitEvent(pipe->d2h, pipe->k_done[c], 0) != cudaSuccess) return SYSCONV_ECUDA;
+        for (int j = 0; j < count; ++j) {
+            const long long n_out = n - q[j] + 1;
+            const long long e1 = o1 < n_out ? o1 : n_out;
+            if (o0 >= e1) continue;
+            if (cudaMemcpyAsync(static_cast<char *>(y_host[j]) + o0 * 4, yd[j] + o0 * 4, (e1 - o0) * 4,
+                                cudaMemcpyDeviceToHost, pipe->d2h) != cudaSuccess) return SYSCONV_ECUDA;
+        }
+    }
+    return pipe->join(s) ? SYSCONV_OK : SYSCONV_ECUDA;
+}
+
 int sysconv2d_host(const void *x_host, int width, int height, const void *w_host, int q, int p, void *y_host,
                    int batch, int dtype, int design, void *workspace_dev, long long workspace_bytes,
                    void *stream)

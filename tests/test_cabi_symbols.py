@@ -26,7 +26,7 @@ def _declared_functions():
 def test_header_declares_the_expected_entry_points():
     names = _declared_functions()
     for must in ("sysconv1d", "sysconv2d", "sysconv1d_strided", "sysconv2d_strided", "sysconv_spacetime_describe",
-                 "sysconv1d_spacetime", "sysconv1d_host", "sysconv2d_host", "sysconv_status_string",
+                 "sysconv1d_spacetime", "sysconv1d_host", "sysconv1d_host_multi", "sysconv2d_host", "sysconv_status_string",
                  "sysconv_design_name", "sysconv_version", "sysconv_launch_count"):
         assert must in names
 
@@ -97,3 +97,26 @@ def test_strided_argument_validation_needs_no_gpu(lib):
     assert b.sysconv2d_strided(x, 64, 64, 64, 0, wi, 3, 3, 2, 2, y, 31, 0, 1, b.U8S8_S32, b.IS, 0) == 2
     w9 = np.ones((9, 9), np.float32)
     assert b.sysconv2d_strided(x, 64, 64, 64, 0, w9, 9, 9, 2, 2, y, 28, 0, 1, b.F32, b.OS, 0) == 2     # beyond 7 x 7
+
+
+def test_host_multi_argument_validation_needs_no_gpu(lib):
+    import ctypes
+    import numpy as np
+    from paper_2010_15884_b200 import binding as b
+    assert b.host_multi_workspace_bytes(1000, [4, 16]) == 4096 + 4096 + 4096
+    assert b.host_multi_workspace_bytes(10, [4, 16]) == -1                       # a filter longer than the signal
+    assert b.host_multi_workspace_bytes(1000, [4], b.U8S8_S32) == -1             # fp32 only
+    w = np.ones(4, np.float32)
+    y = np.zeros(997, np.float32)
+    x = np.zeros(1000, np.float32)
+    q = (ctypes.c_int * 1)(4)
+    d = (ctypes.c_int * 1)(b.OS)
+    wp = (ctypes.c_void_p * 1)(w.ctypes.data)
+    yp = (ctypes.c_void_p * 1)(y.ctypes.data)
+    call = lib.sysconv1d_host_multi
+    vp = ctypes.c_void_p
+    assert call(vp(0), 1000, 1, wp, q, d, yp, b.F32, vp(0x7f0000000000), 1 << 20, vp(0)) == 1          # null x
+    assert call(vp(x.ctypes.data), 1000, 0, wp, q, d, yp, b.F32, vp(0x7f0000000000), 1 << 20, vp(0)) == 1   # no jobs
+    assert call(vp(x.ctypes.data), 1000, 1, wp, q, d, yp, b.F32, vp(0x7f0000000000), 100, vp(0)) == 1       # workspace too small
+    assert call(vp(x.ctypes.data), 1000, 1, wp, q, d, yp, b.F32, vp(0x7f0000000010), 1 << 20, vp(0)) == 1   # misaligned workspace
+    assert call(vp(x.ctypes.data), 1000, 1, wp, q, d, yp, b.U8S8_S32, vp(0x7f0000000000), 1 << 20, vp(0)) == 2

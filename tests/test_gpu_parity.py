@@ -630,6 +630,24 @@ def test_spacetime_executor_rejects_invalid_transforms(cuda_device):
     assert B.sysconv1d_spacetime(x.data_ptr(), 100, w, 5, x.data_ptr(), (1, 0), (0, 1), s0) == 1     # x and y overlap
 
 
+def test_host_multi_entry_point(cuda_device):
+    """One host signal, several (filter, design) jobs in one call: every job's result equals the oracle's."""
+    for n in (3_000_001, 5000, 33):
+        qs = [4, 16, 32, 7, 1]
+        x, ws = inputs.gen_1d_f32(n, qs, seed=123)
+        designs = [B.WS, B.OS, B.IS, B.FSM, B.OS]
+        xh = torch.from_numpy(x).pin_memory()
+        jobs = [(ws[q], d, torch.full((n - q + 1,), CANARY, dtype=torch.float32).pin_memory())
+                for q, d in zip(qs, designs)]
+        work = torch.empty(B.host_multi_workspace_bytes(n, qs), dtype=torch.uint8, device=cuda_device)
+        B.sysconv1d_host_multi(xh, jobs, work)
+        torch.cuda.synchronize()
+        for (w, d, yh), q in zip(jobs, qs):
+            y_ref, s_ref = oracle.conv1d_f32(x, w)
+            assert_close_f32(yh.numpy(), y_ref, s_ref, "n=%d q=%d %s" % (n, q, B.DESIGN_NAMES[d]))
+    assert B.device_status() == 0
+
+
 # ------------------------------------------------------------------------ launches inside a CUDA graph
 
 
