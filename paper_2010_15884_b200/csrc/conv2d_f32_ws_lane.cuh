@@ -109,7 +109,10 @@ conv2d_ws_lane_kernel(const Conv2DArgs a, const __grid_constant__ Taps2D taps, c
 #pragma unroll 1
     for (int j = 0; (j - kGroupDelay) * 8 < n_out; ++j) {
         stage_load(c0 + (j + 1) * kWlChunk);
-#pragma unroll 1
+        // small filters: all eight macro-steps of the chunk unrolled (immediate shared-memory offsets, the reads
+        // of later columns can be issued early); larger ones: two macro-steps per iteration (code size)
+        constexpr int kUnrollU = P * Q <= 25 ? kWlChunk / 2 : 1;
+#pragma unroll kUnrollU
         for (int u = 0; u < kWlChunk / 2; ++u) {
 #pragma unroll
             for (int v = 0; v < 2; ++v) {
