@@ -62,6 +62,55 @@ __device__ __forceinline__ void os_pass_1d_s2(const float *sx, float *so, const 
     }
 }
 
+// ---- OS / FBS, stride 2, paired form for the longer filters (Q >= 12).  PE c at step t and PE c+1 at step
+// t-2 use the SAME input x(2c+t), so the sums of PEs c (even) and c+1 share a 64-bit register pair and ONE
+// packed fp32x2 FMA with the multiplicand (x, x) and the aligned tap pair (w(t), w(t-2)) serves both (the odd
+// PE lags two steps).  Only the even PEs' inputs are needed: x(2c+t) with c = 2m is element 4m+t of the lane
+// block, i.e. four register chains (t mod 4), each moved one pair down every fourth step.  Q+2 steps of 5
+// packed FMAs replace Q steps of 10 scalar ones; the first two and the last two steps touch only one sum
+// of each pair and stay scalar (no zero tap multiplies an input).
+struct Taps1DPairsS2 {
+    float2 p[kMaxQ1 + 2];       // p[t] = (w(t), w(t-2)); taps outside 0..Q-1 are zero
+};
+
+template <int Q>
+__device__ __forceinline__ void os_pass_1d_s2_paired(const float *sx, float *so, const Taps1D &taps,
+                                                     const Taps1DPairsS2 &tp, int lane)
+{
+    constexpr int M = kPeS2 / 2;                // 5 pairs of PEs per lane
+    float X[R1];
+    load_lane_block(sx + lane * R1, X);
+    float S[4][M];                              // S[r][m]: the input pair m uses at the next step t = r mod 4
+#pragma unroll
+    for (int m = 0; m < M; ++m)
+#pragma unroll
+        for (int r = 0; r < 4; ++r) S[r][m] = X[4 * m + r];
+    float2 Z[M];
+#pragma unroll
+    for (int t = 0; t < Q + 2; ++t) {
+        float(&C)[M] = S[t % 4];
+#pragma unroll
+        for (int m = 0; m < M; ++m) {
+            if (t == 0) Z[m] = make_float2(C[m] * taps.w[0], 0.f);
+            else if (t == 1) Z[m].x = fmaf(C[m], taps.w[1], Z[m].x);
+            else if (t >= Q) Z[m].y = fmaf(C[m], taps.w[t - 2], Z[m].y);
+            else Z[m] = __ffma2_rn(make_float2(C[m], C[m]), tp.p[t], Z[m]);
+        }
+        if (t + 4 < Q + 2) {
+            const float in = __shfl_down_sync(kFullMask, C[0], 1);       // lane 31 keeps its own: invalid PEs
+#pragma unroll
+            for (int m = 0; m < M - 1; ++m) C[m] = C[m + 1];
+            C[M - 1] = in;
+        }
+    }
+    // pair m holds y(10 lane + 2m) and y(10 lane + 2m + 1); PEs from 304 on are incomplete
+#pragma unroll
+    for (int m = 0; m < M; ++m) {
+        const int off = lane * kPeS2 + 2 * m;
+        if (off < kWarpOutS2) *reinterpret_cast<float2 *>(so + off) = Z[m];
+    }
+}
+
 template <int Q>
 __device__ __forceinline__ void is_pass_1d_s2(const float *sx, float *so, const Taps1D &taps, int lane)
 {
@@ -91,7 +140,8 @@ __device__ __forceinline__ void is_pass_1d_s2(const float *sx, float *so, const 
 
 template <int DESIGN, int Q, int WARPS, int K>
 __global__ void __launch_bounds__(WARPS *kLanes)
-conv1d_f32_s2_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, unsigned *status_word)
+conv1d_f32_s2_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, const __grid_constant__ Taps1DPairsS2 tpairs,
+                     unsigned *status_word)
 {
     constexpr int kThreads = WARPS * kLanes;
     constexpr int kTileAdv = WARPS * kWarpOut1;         // inputs a tile advances by
@@ -152,7 +202,8 @@ conv1d_f32_s2_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, un
 
             const float *sx = s_in[k] + warp * kWarpOut1;
             float *so = s_out[k] + warp * kWarpOutS2;
-            if (DESIGN == SYSCONV_OS) os_pass_1d_s2<Q>(sx, so, taps, lane);
+            if (DESIGN == SYSCONV_OS && Q >= 12) os_pass_1d_s2_paired<Q>(sx, so, taps, tpairs, lane);
+            else if (DESIGN == SYSCONV_OS) os_pass_1d_s2<Q>(sx, so, taps, lane);
             else is_pass_1d_s2<Q>(sx, so, taps, lane);
 
             if (out_by_copy) {
@@ -180,7 +231,10 @@ cudaError_t launch_conv1d_f32_s2_q(const Conv1DArgs &a, const Taps1D &taps, unsi
     const long long ctas = (a.n_out + per_cta - 1) / per_cta;
     if (ctas > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
     dim3 grid(static_cast<unsigned>(ctas), static_cast<unsigned>(a.batch < 65535 ? a.batch : 65535));
-    conv1d_f32_s2_kernel<DESIGN, Q, WARPS, K><<<grid, WARPS * kLanes, 0, s>>>(a, taps, status_word);
+    Taps1DPairsS2 tp;
+    for (int t = 0; t < kMaxQ1 + 2; ++t)
+        tp.p[t] = make_float2(t < kMaxQ1 ? taps.w[t] : 0.f, t >= 2 ? taps.w[t - 2] : 0.f);
+    conv1d_f32_s2_kernel<DESIGN, Q, WARPS, K><<<grid, WARPS * kLanes, 0, s>>>(a, taps, tp, status_word);
     return cudaGetLastError();
 }
 

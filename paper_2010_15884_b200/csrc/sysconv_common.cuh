@@ -27,12 +27,10 @@ constexpr int R1 = 20;
 constexpr int kWarpIn1 = kLanes * R1;          // 640
 constexpr int kHalo1 = 32;
 constexpr int kWarpOut1 = kWarpIn1 - kHalo1;   // 608
-// weight-stationary arrays, 1-D: sixteen two-lane arrays per warp, each streaming a 76-output segment
-// (76 floats = 19 16-byte words: the broadcast reads of a quarter warp fall in distinct banks)
-constexpr int kWsLanes1 = 2;
-constexpr int kWsArrays1 = kLanes / kWsLanes1;  // 16
+// weight-stationary arrays, 1-D: one array per lane, each streaming a 76-output segment
+// (76 floats = 19 16-byte words: the lanes' 128-bit reads of their own segments fall in distinct banks)
 constexpr int kWsSeg1 = 76;
-// weight-stationary arrays, 2-D: eight four-lane arrays per warp
+// weight-stationary arrays, 2-D, integer data and small problems: eight four-lane arrays per warp
 constexpr int kWsLanes = 4;
 constexpr int kWsArrays = kLanes / kWsLanes;    // 8
 
