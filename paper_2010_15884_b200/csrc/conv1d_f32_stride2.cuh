@@ -138,6 +138,45 @@ __device__ __forceinline__ void is_pass_1d_s2(const float *sx, float *so, const 
     }
 }
 
+// ---- IS / SBM, stride 2, paired form for the longer filters (Q >= 12).  The sums of outputs c (even) and
+// c+1 start two PEs apart and travel together in one 64-bit register pair: PE s adds x(s)*w(t) to the first
+// and x(s)*w(t-2) to the second, t = s-2c, with ONE packed fp32x2 FMA.  The pair sits in PE 2c+t at step t,
+// so every fourth PE holds a live pair: Q+2 steps of 5 packed FMAs, lane-to-lane transfer every fourth step.
+template <int Q>
+__device__ __forceinline__ void is_pass_1d_s2_paired(const float *sx, float *so, const Taps1D &taps,
+                                                     const Taps1DPairsS2 &tp, int lane)
+{
+    float X[R1];
+    load_lane_block(sx + lane * R1, X);
+    constexpr int M = R1 / 4;                   // 5 live pairs per lane
+    float2 P[4][M];                             // P[r][i]: the pair in PE 4i+r, live while r = t mod 4
+#pragma unroll
+    for (int t = 0; t < Q + 2; ++t) {
+        const int r = t % 4;
+        float2 up = make_float2(0.f, 0.f);
+        if (t > 0 && r == 0)                    // lane 0 keeps its own: invalid PEs
+            up = make_float2(__shfl_up_sync(kFullMask, P[3][M - 1].x, 1), __shfl_up_sync(kFullMask, P[3][M - 1].y, 1));
+#pragma unroll
+        for (int i = M - 1; i >= 0; --i) {
+            const float x = X[4 * i + r];
+            float2 prev = up;
+            if (r > 0) prev = P[r - 1][i];
+            else if (i > 0) prev = P[3][i - 1];
+            if (t == 0) P[r][i] = make_float2(x * taps.w[0], 0.f);
+            else if (t == 1) P[r][i] = make_float2(fmaf(x, taps.w[1], prev.x), prev.y);
+            else if (t >= Q) P[r][i] = make_float2(prev.x, fmaf(x, taps.w[t - 2], prev.y));
+            else P[r][i] = __ffma2_rn(make_float2(x, x), tp.p[t], prev);
+        }
+    }
+    // PE s (s = Q+1 mod 4) holds y((s-Q-1)/2) and the next output; the first PEs of the slice hold incomplete sums
+    constexpr int rl = (Q + 1) % 4;
+#pragma unroll
+    for (int i = 0; i < M; ++i) {
+        const int start = lane * R1 + 4 * i + rl - (Q + 1);
+        if (start >= 0 && start < 2 * kWarpOutS2) *reinterpret_cast<float2 *>(so + (start >> 1)) = P[rl][i];
+    }
+}
+
 template <int DESIGN, int Q, int WARPS, int K>
 __global__ void __launch_bounds__(WARPS *kLanes)
 conv1d_f32_s2_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, const __grid_constant__ Taps1DPairsS2 tpairs,
@@ -204,6 +243,7 @@ conv1d_f32_s2_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, co
             float *so = s_out[k] + warp * kWarpOutS2;
             if (DESIGN == SYSCONV_OS && Q >= 12) os_pass_1d_s2_paired<Q>(sx, so, taps, tpairs, lane);
             else if (DESIGN == SYSCONV_OS) os_pass_1d_s2<Q>(sx, so, taps, lane);
+            else if (Q >= 12) is_pass_1d_s2_paired<Q>(sx, so, taps, tpairs, lane);
             else is_pass_1d_s2<Q>(sx, so, taps, lane);
 
             if (out_by_copy) {
