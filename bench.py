@@ -11,7 +11,8 @@ launches per step); the metric is output elements per second.
 
 * value      device-resident inputs, CUDA-event time around K steps
 * e2e        the same step through the host-buffer C-ABI entry points (pinned
-             host memory, host<->device copies inside the timed region)
+             host memory, host<->device copies inside the timed region); 1-D:
+             one sysconv1d_host_multi call per step (signal copied in once)
 * roofline   the kernel with the largest share of the step, algorithmic bytes /
              its average launch time (per-launch CUDA events) vs the measured
              HBM copy bandwidth of this machine (MEASURED_PEAKS.json)
