@@ -464,6 +464,10 @@ def run_ours(args):
                 "value": round(outs / secs / 1e9, 4), "unit": "Gpix/s", "cores": cores, "kind": "oracle",
                 "sample": "%s of configuration %d (%.1f s wall on %d threads)" % (what, cfg_id, secs, cores)}
         line["per_kernel"] = detail_rows(cases, hbm_gbs, peak_kind, sm_max)
+        # context only: another machine, another baseline (Intel GEN9.5, fixed-function sampler); not comparable
+        line["paper_context"] = ("the paper (abstract, Section 6) reports its best software systolic designs, SBM and "
+                                 "FBS, 14-59 % faster than the GEN9.5 GPU's hardware sampler on the same 1-D and "
+                                 "small 2-D convolutions; neither that GPU nor a sampler exists here")
         if not args.no_detail and world == 1:
             del cases, keep
             torch.cuda.empty_cache()
