@@ -183,6 +183,175 @@ cudaError_t launch_conv2d_u8_os_dp4a(const Conv2DArgs &a, const Taps2DInt &t, cu
     return cudaGetLastError();
 }
 
+// ---------------------------------------------------------------------------
+// IS / SBM on the packed integer datapath, filters up to 7 rows.  A word-PE keeps four consecutive pixels of
+// each of the P input rows of the window, together with the three words that start 1, 2 and 3 pixels later
+// (built once per input row with PRMT from the next PE's word): the stationary inputs.  The sums of the four
+// outputs 4k .. 4k+3 start in word-PE k and move one word-PE up per step; a step applies FOUR taps of each of
+// the P filter rows with dp4a, so a pass is ceil(Q/4) steps and the four sums end up 128-bit aligned in
+// word-PE k + ceil(Q/4) - 1 without any drain.  A strip is two runs of 32 words (lane l holds word l of each
+// run: contiguous loads and stores), its last word-PE has no right neighbour and its first ones no left
+// neighbour, so a strip yields 4*(64 - ceil(Q/4)) outputs and consecutive strips overlap by ceil(Q/4) words.
+// ---------------------------------------------------------------------------
+template <int Q>
+struct IsDp4aGeom {
+    static constexpr int G = (Q + 3) / 4;
+    static constexpr int kValid = 4 * (64 - G);         // outputs per strip
+};
+
+template <int P, int Q>
+__global__ void __launch_bounds__(kThreads2)
+conv2d_u8_is_dp4a_kernel(const Conv2DArgs a, const __grid_constant__ TapsPacked taps, const int band_h)
+{
+    constexpr int G = IsDp4aGeom<Q>::G;
+    constexpr int kValid = IsDp4aGeom<Q>::kValid;
+    const int lane = threadIdx.x & (kLanes - 1);
+    const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;
+    const int c0 = strip * kValid;              // first output column = first input column of the strip
+    if (c0 >= a.out_w) return;
+    const int r0 = blockIdx.y * band_h;
+    const int r1 = min(r0 + band_h, a.out_h);
+    const uint8_t *xb = static_cast<const uint8_t *>(a.x) + blockIdx.z * a.x_bstride;
+    int *yb = static_cast<int *>(a.y) + blockIdx.z * a.y_bstride;
+    const int y_align = row_alignment(static_cast<const int *>(a.y), a.y_pitch, a.y_bstride, a.batch);
+    const int oend = min(a.out_w, c0 + kValid);
+
+    // the lane's two words of one input row (pixels beyond the image read as zero)
+    auto fetch = [&](int row, unsigned (&w)[2]) {
+        const uint8_t *rowp = xb + static_cast<long long>(min(row, a.height - 1)) * a.x_pitch;
+#pragma unroll
+        for (int n = 0; n < 2; ++n) {
+            const int c = c0 + 4 * (kLanes * n + lane);
+            unsigned v = 0;
+            if (c + 4 <= a.width) {
+                v = __ldg(reinterpret_cast<const unsigned *>(rowp + c));
+            } else {
+#pragma unroll
+                for (int e = 0; e < 3; ++e)
+                    if (c + e < a.width) v |= static_cast<unsigned>(rowp[c + e]) << (8 * e);
+            }
+            w[n] = v;
+        }
+    };
+    // the four stationary words of both word-PEs for one input row
+    auto expand = [&](const unsigned (&w)[2], unsigned (&s)[2][4]) {
+        // the next PE's word: the next lane's, and for lane 31 of run 0 the first word of run 1
+        const unsigned send = lane == 0 ? w[1] : w[0];
+        const unsigned n0 = __shfl_sync(kFullMask, send, (lane + 1) & (kLanes - 1));
+        const unsigned n1 = __shfl_down_sync(kFullMask, w[1], 1);    // the strip's last PE keeps its own: invalid sums
+        const unsigned nx[2] = {n0, n1};
+#pragma unroll
+        for (int n = 0; n < 2; ++n) {
+            s[n][0] = w[n];
+            s[n][1] = __byte_perm(w[n], nx[n], 0x4321);
+            s[n][2] = __byte_perm(w[n], nx[n], 0x5432);
+            s[n][3] = __byte_perm(w[n], nx[n], 0x6543);
+        }
+    };
+
+    unsigned S[P][2][4];                        // PE registers: rows r .. r+P-1
+#pragma unroll
+    for (int p = 0; p < P; ++p)
+#pragma unroll
+        for (int n = 0; n < 2; ++n)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) S[p][n][i] = 0;
+#pragma unroll
+    for (int p = 0; p < P - 1; ++p) {
+        unsigned w[2];
+        fetch(r0 + p, w);
+        expand(w, S[p + 1]);
+    }
+    unsigned nW[2];
+    fetch(r0 + P - 1, nW);
+
+#pragma unroll 1
+    for (int r = r0; r < r1; ++r) {
+        // the window of input rows slides down by one
+#pragma unroll
+        for (int p = 0; p < P - 1; ++p)
+#pragma unroll
+            for (int n = 0; n < 2; ++n)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) S[p][n][i] = S[p + 1][n][i];
+        expand(nW, S[P - 1]);
+        if (r + 1 < r1) fetch(r + P, nW);
+
+        int Z[2][4];
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                int z0 = 0, z1 = 0;
+                if (g > 0) {
+                    // the sums move one word-PE up: run 0 from the previous lane, run 1 likewise, its first PE
+                    // from the last PE of run 0 (the strip's first PE has no left neighbour: invalid sums)
+                    const int send = lane == kLanes - 1 ? Z[0][i] : Z[1][i];
+                    z0 = __shfl_up_sync(kFullMask, Z[0][i], 1);
+                    z1 = __shfl_sync(kFullMask, send, (lane - 1) & (kLanes - 1));
+                }
+#pragma unroll
+                for (int p = 0; p < P; ++p) {
+                    z0 = dp4a_u8s8(S[p][0][i], taps.w[p * 4 + g], z0);
+                    z1 = dp4a_u8s8(S[p][1][i], taps.w[p * 4 + g], z1);
+                }
+                Z[0][i] = z0;
+                Z[1][i] = z1;
+            }
+        }
+        // word-PE k holds the outputs that started in word-PE k - (G-1)
+        int *orow = yb + static_cast<long long>(r) * a.y_pitch;
+#pragma unroll
+        for (int n = 0; n < 2; ++n) {
+            const int k = kLanes * n + lane - (G - 1);
+            if (k >= 0) store_group<U8Traits>(orow, c0 + 4 * k, oend, y_align, Z[n]);
+        }
+    }
+}
+
+template <int P, int Q>
+cudaError_t launch_conv2d_u8_is_dp4a(const Conv2DArgs &a, const Taps2DInt &t, cudaStream_t s)
+{
+    TapsPacked pk;
+    for (int p = 0; p < kMaxP2; ++p)
+        for (int g = 0; g < 4; ++g) {
+            unsigned v = 0;
+            for (int e = 0; e < 4; ++e) {
+                const int q = 4 * g + e;
+                const int w = (p < P && q < Q) ? t.w[p * Q + q] : 0;
+                v |= (static_cast<unsigned>(w) & 0xffu) << (8 * e);
+            }
+            pk.w[p * 4 + g] = static_cast<int>(v);
+        }
+    const int strips = (a.out_w + IsDp4aGeom<Q>::kValid - 1) / IsDp4aGeom<Q>::kValid;
+    const long long warps = static_cast<long long>(strips) * a.batch;
+    const long long bands = (148LL * 32 + warps - 1) / warps;
+    long long h = (a.out_h + bands - 1) / bands;
+    const long long lo = 2 * P > 8 ? 2 * P : 8;         // the first P-1 rows of a band are loaded twice
+    if (h > 64) h = 64;
+    if (h < lo) h = lo;
+    const long long fit = (a.out_h + 65534LL) / 65535;  // grid.y limit
+    if (h < fit) h = fit;
+    const int band_h = static_cast<int>(h);
+    dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + band_h - 1) / band_h, a.batch);
+    conv2d_u8_is_dp4a_kernel<P, Q><<<grid, kThreads2, 0, s>>>(a, pk, band_h);
+    return cudaGetLastError();
+}
+
+template <int P, int Q>
+struct FastPath2D<U8Traits, SYSCONV_IS, P, Q> {
+    static bool launch(const Conv2DArgs &a, const Taps2DInt &taps, cudaStream_t s, cudaError_t *err)
+    {
+        if constexpr (P <= 7) {
+            if (!u8_dp4a_eligible(a)) return false;
+            *err = launch_conv2d_u8_is_dp4a<P, Q>(a, taps, s);
+            return true;
+        } else {
+            return false;
+        }
+    }
+};
+
 // uint8 rows that start 4-byte aligned run on the packed (dp4a) kernel
 template <int P, int Q>
 struct FastPath2D<U8Traits, SYSCONV_OS, P, Q> {

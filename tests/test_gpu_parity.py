@@ -700,22 +700,24 @@ def test_2d_u8_shapes_and_extremes(cuda_device, design, pq):
         check_2d(xm, np.full(pq, v, np.int8), design, cuda_device)
 
 
-@pytest.mark.parametrize("pq", [(1, 1), (3, 3), (5, 5), (7, 7), (7, 15), (8, 15), (15, 15), (9, 2), (4, 13), (12, 8)],
-                         ids=lambda f: "%dx%d" % f)
-def test_2d_u8_os_packed_rows(cuda_device, pq):
-    """Rows that start 16-byte aligned take the packed four-taps-per-step kernel: several strips, a ragged
-    right edge, pitch padding, unaligned outputs, and the extreme pixel/tap values."""
+@pytest.mark.parametrize("design", [B.OS, B.IS], ids=_ids)
+@pytest.mark.parametrize("pq", [(1, 1), (3, 3), (5, 5), (7, 7), (7, 15), (8, 15), (15, 15), (9, 2), (4, 13), (12, 8),
+                                (1, 4), (2, 5), (6, 9), (7, 12), (3, 8)], ids=lambda f: "%dx%d" % f)
+def test_2d_u8_packed_rows(cuda_device, design, pq):
+    """Rows that start 4-byte aligned take the packed four-taps-per-step kernels (OS: every filter size; IS: up to
+    seven filter rows): several strips, a ragged right edge, pitch padding, unaligned outputs, and the extreme
+    pixel/tap values."""
     p, q = pq
     x, ws = inputs.gen_2d_u8s8(1101, 41, [pq], seed=90 + p + q, batch=2)
-    check_2d(x, ws[pq], B.OS, cuda_device, x_pitch=1104)
-    check_2d(x, ws[pq], B.OS, cuda_device, x_pitch=1120, y_pitch=1103, y_off=3)
-    check_2d(x[:, :, :1040], ws[pq], B.OS, cuda_device)
-    check_2d(x[:, :, :528], ws[pq], B.OS, cuda_device, x_pitch=528)
+    check_2d(x, ws[pq], design, cuda_device, x_pitch=1104)
+    check_2d(x, ws[pq], design, cuda_device, x_pitch=1120, y_pitch=1103, y_off=3)
+    check_2d(x[:, :, :1040], ws[pq], design, cuda_device)
+    check_2d(x[:, :, :528], ws[pq], design, cuda_device, x_pitch=528)
     xm = np.full((1, 33, 160), 255, np.uint8)
     for v in (127, -128):
-        check_2d(xm, np.full(pq, v, np.int8), B.OS, cuda_device)
+        check_2d(xm, np.full(pq, v, np.int8), design, cuda_device)
     wmix = np.where((np.arange(p * q).reshape(p, q) % 2) == 0, 127, -128).astype(np.int8)
-    check_2d(x[:1, :, :512], wmix, B.OS, cuda_device)
+    check_2d(x[:1, :, :512], wmix, design, cuda_device)
 
 
 @pytest.mark.parametrize("design", DESIGNS, ids=_ids)
