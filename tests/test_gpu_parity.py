@@ -797,3 +797,81 @@ def test_unsupported_and_invalid_on_device(cuda_device):
     before = B.launch_count()
     B.conv1d(x, np.ones(8, np.float32))
     assert B.launch_count() == before + 1
+
+
+# ------------------------------------------------------------------------ randomized shapes
+
+
+def test_randomized_1d_shapes(cuda_device):
+    """Seeded random lengths, filter lengths, designs, strides, batches and pointer offsets."""
+    rng = np.random.default_rng(2024)
+    for case in range(160):
+        q = int(rng.integers(1, 33))
+        n = q + int(rng.choice([0, 1, 2, 5, 100, 607, 608, 609, 1215, 1216, 1217, 2431, 2432, 2433, 4000, 9000]))
+        n += int(rng.integers(0, 40))
+        batch = int(rng.choice([1, 1, 2, 3]))
+        stride = int(rng.choice([1, 1, 2]))
+        design = int(rng.choice([B.OS, B.IS] if stride == 2 else [B.WS, B.OS, B.IS, B.FSM, B.BFS, B.FFS]))
+        x_off, y_off = int(rng.integers(0, 4)), int(rng.integers(0, 4))
+        xs = n + int(rng.integers(0, 5)) * (batch > 1)
+        n_out = (n - q) // stride + 1
+        ys = n_out + int(rng.integers(0, 5)) * (batch > 1)
+        x = rng.uniform(-1, 1, (batch, n)).astype(np.float32)
+        w = rng.uniform(-1, 1, q).astype(np.float32)
+        xb = torch.zeros(x_off + batch * xs + 8, dtype=torch.float32, device=cuda_device)
+        yb = torch.full((y_off + batch * ys + 8,), CANARY, dtype=torch.float32, device=cuda_device)
+        xb[x_off: x_off + batch * xs].view(batch, xs)[:, :n] = torch.from_numpy(x).to(cuda_device)
+        st = B.sysconv1d_strided(xb.data_ptr() + 4 * x_off, n, xs, w, q, stride, yb.data_ptr() + 4 * y_off, ys, batch,
+                                 B.F32, design, torch.cuda.current_stream().cuda_stream)
+        what = "case %d: n=%d q=%d batch=%d stride=%d design=%d offs=%d,%d" % (case, n, q, batch, stride, design, x_off, y_off)
+        assert st == 0, what
+        torch.cuda.synchronize()
+        yh = yb.cpu().numpy()
+        body = yh[y_off: y_off + batch * ys].reshape(batch, ys)
+        assert (body[:, n_out:] == CANARY).all() and (yh[:y_off] == CANARY).all(), what
+        assert (yh[y_off + batch * ys:] == CANARY).all(), what
+        for b in range(batch):
+            y_ref, s_ref = oracle.conv1d_f32_strided(x[b], w, stride)
+            assert_close_f32(body[b, :n_out], y_ref, s_ref, what)
+    assert B.device_status() == 0
+
+
+def test_randomized_2d_shapes(cuda_device):
+    """Seeded random image sizes (around the strip widths of every kernel), filters, designs, data types,
+    strides, pitches and offsets."""
+    rng = np.random.default_rng(2025)
+    edges = [1, 2, 3, 4, 5, 31, 32, 33, 119, 120, 121, 124, 125, 127, 128, 129, 236, 240, 244, 248, 249, 252, 253,
+             255, 256, 257, 480, 496, 504, 511, 512, 513, 600, 1000]
+    for case in range(220):
+        p, q = int(rng.integers(1, 16)), int(rng.integers(1, 16))
+        is_u8 = bool(rng.integers(0, 3) == 0)
+        stride = 1 if is_u8 else int(rng.choice([1, 1, 2]))
+        if stride == 2:
+            p, q = min(p, 7), min(q, 7)
+        design = int(rng.choice([B.OS, B.IS] if stride == 2 else [B.WS, B.OS, B.IS]))
+        ow = int(rng.choice(edges)) + int(rng.integers(0, 3))
+        oh = int(rng.choice([1, 2, 7, 8, 9, 15, 16, 17, 31, 33, 64, 70]))
+        wd, h = stride * (ow - 1) + q + int(rng.integers(0, stride)), stride * (oh - 1) + p + int(rng.integers(0, stride))
+        batch = int(rng.choice([1, 1, 2]))
+        aligned = bool(rng.integers(0, 2))
+        x_pitch = (wd + 3) // 4 * 4 if aligned else wd + int(rng.integers(0, 4))
+        x_off = 0 if aligned else int(rng.integers(0, 4))
+        y_pitch = ow + int(rng.integers(0, 4))
+        y_off = int(rng.integers(0, 4))
+        what = "case %d: %dx%d image, %dx%d filter, batch %d, %s, stride %d, design %d, pitches %d/%d, offs %d/%d" % (
+            case, wd, h, p, q, batch, "u8" if is_u8 else "f32", stride, design, x_pitch, y_pitch, x_off, y_off)
+        if is_u8:
+            x = rng.integers(0, 256, (batch, h, wd)).astype(np.uint8)
+            w = rng.integers(-128, 128, (p, q)).astype(np.int8)
+            check_2d(x, w, design, cuda_device, x_pitch=x_pitch, y_pitch=y_pitch, x_off=x_off, y_off=y_off)
+        else:
+            x = rng.random((batch, h, wd), dtype=np.float32)
+            w = rng.uniform(-1, 1, (p, q)).astype(np.float32)
+            try:
+                if stride == 2:
+                    check_2d_s2(x, w, design, cuda_device, x_pitch=x_pitch, y_pitch=y_pitch, x_off=x_off, y_off=y_off)
+                else:
+                    check_2d(x, w, design, cuda_device, x_pitch=x_pitch, y_pitch=y_pitch, x_off=x_off, y_off=y_off)
+            except AssertionError as e:
+                raise AssertionError(what + ": " + str(e))
+    assert B.device_status() == 0
