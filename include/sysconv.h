@@ -123,7 +123,7 @@ int sysconv2d(const void *x_dev, int width, int height, long long x_pitch, long 
  * ((height-p)/stride_r + 1) x ((width-q)/stride_c + 1) outputs per image (Section 5 runs the strided
  * design row by row).  All other arguments as for sysconv1d / sysconv2d.
  * Stride 1 is the unstrided call.  Stride 2 (both directions in 2-D) is built for fp32 data, the
- * SYSCONV_OS and SYSCONV_IS designs, q <= 32 in 1-D and p, q <= 7 in 2-D; every other combination returns
+ * SYSCONV_OS and SYSCONV_IS designs, q <= 32 in 1-D and p, q <= 7 and batch <= 65535 in 2-D; every other combination returns
  * SYSCONV_EUNSUPPORTED (strides below 1: SYSCONV_EINVAL).
  */
 int sysconv1d_strided(const void *x_dev, long long n, long long x_batch_stride,

@@ -108,8 +108,28 @@ bool overlaps(const void *a, unsigned long long an, const void *b, unsigned long
     return pa < pb + bn && pb < pa + an;
 }
 
+int dispatch2d_once(const sysconv::Conv2DArgs &a, const void *w_host, int q, int p, int dtype, int design,
+                    cudaStream_t s);
+
+// The image index is a grid dimension (at most 65535): larger batches go out in slices, one launch each.
+constexpr int kMaxBatchPerLaunch = 65535;
 int dispatch2d(const sysconv::Conv2DArgs &a, const void *w_host, int q, int p, int dtype, int design,
                cudaStream_t s)
+{
+    if (a.batch <= kMaxBatchPerLaunch) return dispatch2d_once(a, w_host, q, p, dtype, design, s);
+    for (int b0 = 0; b0 < a.batch; b0 += kMaxBatchPerLaunch) {
+        sysconv::Conv2DArgs part = a;
+        part.batch = a.batch - b0 < kMaxBatchPerLaunch ? a.batch - b0 : kMaxBatchPerLaunch;
+        part.x = static_cast<const char *>(a.x) + static_cast<long long>(b0) * a.x_bstride * (long long)in_elt_bytes(dtype);
+        part.y = static_cast<char *>(a.y) + static_cast<long long>(b0) * a.y_bstride * 4LL;
+        const int st = dispatch2d_once(part, w_host, q, p, dtype, design, s);
+        if (st != SYSCONV_OK) return st;
+    }
+    return SYSCONV_OK;
+}
+
+int dispatch2d_once(const sysconv::Conv2DArgs &a, const void *w_host, int q, int p, int dtype, int design,
+                    cudaStream_t s)
 {
     using namespace sysconv;
     int launches = 0;
@@ -225,7 +245,7 @@ int sysconv2d_strided(const void *x_dev, int width, int height, long long x_pitc
     const unsigned long long x_bytes = ((unsigned long long)(batch - 1) * x_batch_stride + x_img) * in_elt_bytes(dtype);
     const unsigned long long y_bytes = ((unsigned long long)(batch - 1) * y_batch_stride + y_img) * 4ull;
     if (overlaps(x_dev, x_bytes, y_dev, y_bytes)) return SYSCONV_EINVAL;
-    if (stride_c != 2 || stride_r != 2 || dtype != SYSCONV_F32) return SYSCONV_EUNSUPPORTED;
+    if (stride_c != 2 || stride_r != 2 || dtype != SYSCONV_F32 || batch > 65535) return SYSCONV_EUNSUPPORTED;
     if (design != SYSCONV_OS && design != SYSCONV_IS) return SYSCONV_EUNSUPPORTED;
     Conv2DArgs a;
     a.x = x_dev; a.y = y_dev;

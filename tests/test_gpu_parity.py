@@ -799,6 +799,26 @@ def test_unsupported_and_invalid_on_device(cuda_device):
     assert B.launch_count() == before + 1
 
 
+def test_2d_batches_beyond_one_grid(cuda_device):
+    """More images than one launch can index (65535): the call goes out in slices."""
+    batch = 65535 + 4097
+    rng = np.random.default_rng(12)
+    picks = [0, 1, 65534, 65535, 65536, batch - 1]
+    x = rng.random((batch, 6, 9), dtype=np.float32)
+    w = rng.uniform(-1, 1, (3, 2)).astype(np.float32)
+    xu = rng.integers(0, 256, (batch, 6, 12)).astype(np.uint8)
+    wu = rng.integers(-128, 128, (2, 5)).astype(np.int8)
+    for design in DESIGNS:
+        y = B.conv2d(torch.from_numpy(x).to(cuda_device), w, design).cpu().numpy()
+        yu = B.conv2d(torch.from_numpy(xu).to(cuda_device), wu, design).cpu().numpy()
+        for b in picks:
+            y_ref, s_ref = oracle.conv2d_f32(x[b], w)
+            assert_close_f32(y[b], y_ref, s_ref, "image %d" % b)
+            np.testing.assert_array_equal(yu[b], oracle.conv2d_u8s8_s32(xu[b], wu))
+    st = B.sysconv2d_strided(1 << 20, 9, 6, 9, 54, w, 2, 3, 2, 2, 1 << 30, 4, 8, batch, B.F32, B.OS, 0)
+    assert st == 2
+
+
 # ------------------------------------------------------------------------ randomized shapes
 
 
