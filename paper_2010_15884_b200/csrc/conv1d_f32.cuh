@@ -48,11 +48,11 @@ struct DefaultShape1D {
 
 // ---- ordinary-load staging (ragged or unaligned tiles) ------------------------
 
-// Copy x[t0 .. t0 + tile_in) to shared memory, zeros beyond the signal's end.
+// Copy x[t0 + first .. t0 + tile_in) to shared memory, zeros beyond the signal's end.
 __device__ __forceinline__ void stage_in_1d(const float *__restrict__ xg, long long n, long long t0,
-                                            float *s_in, int tile_in, int threads)
+                                            float *__restrict__ s_in, int tile_in, int threads, int first = 0)
 {
-    for (int i = threadIdx.x; i < tile_in; i += threads) {
+    for (int i = first + threadIdx.x; i < tile_in; i += threads) {
         const long long g = t0 + i;
         s_in[i] = g < n ? xg[g] : 0.f;
     }
@@ -414,6 +414,13 @@ conv1d_f32_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, const
         for (int k = 0; k < K; ++k) mbar_init(&full[k], 1);
         mbar_init_fence();
     }
+    // elements of tile k that arrive by bulk copy: the part of the tile inside the signal, in whole 16-byte words
+    auto bulk_in = [&](int k) -> int {
+        const long long t0 = base + k * G::kTileOut;
+        if (!x_ok || t0 >= a.n) return 0;
+        const long long valid = a.n - t0 < G::kTileIn ? a.n - t0 : G::kTileIn;
+        return static_cast<int>(valid) & ~3;
+    };
     unsigned phase = 0;
     for (int b = blockIdx.y; b < a.batch; b += gridDim.y) {
         const float *xg = static_cast<const float *>(a.x) + b * a.x_bstride;
@@ -423,10 +430,10 @@ conv1d_f32_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, const
         if (threadIdx.x == 0) {
 #pragma unroll
             for (int k = 0; k < K; ++k) {
-                const long long t0 = base + k * G::kTileOut;
-                if (x_ok && t0 + G::kTileIn <= a.n) {
-                    mbar_arrive_expect_tx(&full[k], G::kTileIn * 4);
-                    bulk_load(s_in[k], xg + t0, G::kTileIn * 4, &full[k]);
+                const int be = bulk_in(k);
+                if (be > 0) {
+                    mbar_arrive_expect_tx(&full[k], be * 4);
+                    bulk_load(s_in[k], xg + (base + k * G::kTileOut), be * 4, &full[k]);
                 }
             }
         }
@@ -434,23 +441,25 @@ conv1d_f32_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, const
         for (int k = 0; k < K; ++k) {
             const long long t0 = base + k * G::kTileOut;
             if (t0 >= a.n_out) break;
-            const bool in_by_copy = x_ok && t0 + G::kTileIn <= a.n;
-            const bool out_by_copy = y_ok && t0 + G::kTileOut <= a.n_out;
-            if (in_by_copy) {
+            const int be = bulk_in(k);
+            if (be > 0) {
                 const bool ok = mbar_wait_bounded(&full[k], phase);
                 const bool give_up = WARPS == 1 ? __any_sync(kFullMask, !ok) != 0 : __syncthreads_or(!ok) != 0;
                 if (give_up) {
                     if (threadIdx.x == 0) {
                         atomicExch(status_word, 1u);
                         for (int j = k + 1; j < K; ++j)      // copies still in flight target this CTA's memory
-                            if (x_ok && base + j * G::kTileOut + G::kTileIn <= a.n)
-                                mbar_wait_bounded(&full[j], phase, 1u << 16);
+                            if (bulk_in(j) > 0) mbar_wait_bounded(&full[j], phase, 1u << 16);
                         bulk_wait_read<0>();
                     }
                     return;
                 }
-            } else {
-                stage_in_1d(xg, a.n, t0, s_in[k], G::kTileIn, G::kThreads);
+            }
+            if (be < G::kTileIn) {
+                // ragged last tile or unaligned signal: the rest by ordinary loads, zeros beyond the signal's end
+                // (two call sites: with a literal start the loop's trip count is known and its loads are issued together)
+                if (be == 0) stage_in_1d(xg, a.n, t0, s_in[k], G::kTileIn, G::kThreads);
+                else stage_in_1d(xg, a.n, t0, s_in[k], G::kTileIn, G::kThreads, be);
                 __syncthreads();
             }
 
@@ -465,13 +474,19 @@ conv1d_f32_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, const
             else if (DESIGN == SYSCONV_BFS) bfs_pass_1d<Q>(sx, so, taps, lane);
             else ffs_pass_1d<Q>(sx, so, taps, lane);
 
-            if (out_by_copy) {
+            if (y_ok) {
+                // the warp's outputs inside the signal: whole 16-byte words by bulk store, up to three more by lanes
+                const long long w0 = t0 + warp * G::kWarpOut;
+                long long vw = a.n_out - w0;
+                vw = vw > G::kWarpOut ? G::kWarpOut : (vw < 0 ? 0 : vw);
+                const int bo = static_cast<int>(vw) & ~3;
                 fence_proxy_async();                     // my shared-memory writes, before the bulk store reads them
                 __syncwarp();
-                if (lane == 0) {
-                    bulk_store(yg + t0 + warp * G::kWarpOut, so, G::kWarpOut * 4);
+                if (lane == 0 && bo > 0) {
+                    bulk_store(yg + w0, so, bo * 4);
                     bulk_commit();
                 }
+                if (bo + lane < vw) yg[w0 + bo + lane] = so[bo + lane];
             } else {
                 __syncthreads();
                 stage_out_1d(yg, a.n_out, t0, s_out[k], G::kTileOut, G::kThreads);
