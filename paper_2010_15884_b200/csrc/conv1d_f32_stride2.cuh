@@ -199,6 +199,13 @@ conv1d_f32_s2_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, co
         for (int k = 0; k < K; ++k) mbar_init(&full[k], 1);
         mbar_init_fence();
     }
+    // elements of tile k that arrive by bulk copy: the part of the tile inside the signal, in whole 16-byte words
+    auto bulk_in = [&](int k) -> int {
+        const long long t0 = base_in + k * kTileAdv;
+        if (!x_ok || t0 >= a.n) return 0;
+        const long long valid = a.n - t0 < kTileIn ? a.n - t0 : kTileIn;
+        return static_cast<int>(valid) & ~3;
+    };
     unsigned phase = 0;
     for (int b = blockIdx.y; b < a.batch; b += gridDim.y) {
         const float *xg = static_cast<const float *>(a.x) + b * a.x_bstride;
@@ -207,10 +214,10 @@ conv1d_f32_s2_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, co
         if (threadIdx.x == 0) {
 #pragma unroll
             for (int k = 0; k < K; ++k) {
-                const long long t0 = base_in + k * kTileAdv;
-                if (x_ok && t0 + kTileIn <= a.n) {
-                    mbar_arrive_expect_tx(&full[k], kTileIn * 4);
-                    bulk_load(s_in[k], xg + t0, kTileIn * 4, &full[k]);
+                const int be = bulk_in(k);
+                if (be > 0) {
+                    mbar_arrive_expect_tx(&full[k], be * 4);
+                    bulk_load(s_in[k], xg + (base_in + k * kTileAdv), be * 4, &full[k]);
                 }
             }
         }
@@ -219,23 +226,24 @@ conv1d_f32_s2_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, co
             const long long t0 = base_in + k * kTileAdv;    // first input of the tile (even)
             const long long o0 = t0 / 2;                    // first output of the tile
             if (o0 >= a.n_out) break;
-            const bool in_by_copy = x_ok && t0 + kTileIn <= a.n;
-            const bool out_by_copy = y_ok && o0 + kTileOut <= a.n_out;
-            if (in_by_copy) {
+            const int be = bulk_in(k);
+            if (be > 0) {
                 const bool ok = mbar_wait_bounded(&full[k], phase);
                 const bool give_up = WARPS == 1 ? __any_sync(kFullMask, !ok) != 0 : __syncthreads_or(!ok) != 0;
                 if (give_up) {
                     if (threadIdx.x == 0) {
                         atomicExch(status_word, 1u);
                         for (int j = k + 1; j < K; ++j)      // copies still in flight target this CTA's memory
-                            if (x_ok && base_in + j * kTileAdv + kTileIn <= a.n)
-                                mbar_wait_bounded(&full[j], phase, 1u << 16);
+                            if (bulk_in(j) > 0) mbar_wait_bounded(&full[j], phase, 1u << 16);
                         bulk_wait_read<0>();
                     }
                     return;
                 }
-            } else {
-                stage_in_1d(xg, a.n, t0, s_in[k], kTileIn, kThreads);
+            }
+            if (be < kTileIn) {
+                // ragged last tile or unaligned signal: the rest by ordinary loads, zeros beyond the signal's end
+                if (be == 0) stage_in_1d(xg, a.n, t0, s_in[k], kTileIn, kThreads);
+                else stage_in_1d(xg, a.n, t0, s_in[k], kTileIn, kThreads, be);
                 __syncthreads();
             }
 
@@ -246,13 +254,19 @@ conv1d_f32_s2_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, co
             else if (Q >= 12) is_pass_1d_s2_paired<Q>(sx, so, taps, tpairs, lane);
             else is_pass_1d_s2<Q>(sx, so, taps, lane);
 
-            if (out_by_copy) {
+            if (y_ok) {
+                // the warp's outputs inside the signal: whole 16-byte words by bulk store, up to three more by lanes
+                const long long w0 = o0 + warp * kWarpOutS2;
+                long long vw = a.n_out - w0;
+                vw = vw > kWarpOutS2 ? kWarpOutS2 : (vw < 0 ? 0 : vw);
+                const int bo = static_cast<int>(vw) & ~3;
                 fence_proxy_async();
                 __syncwarp();
-                if (lane == 0) {
-                    bulk_store(yg + o0 + warp * kWarpOutS2, so, kWarpOutS2 * 4);
+                if (lane == 0 && bo > 0) {
+                    bulk_store(yg + w0, so, bo * 4);
                     bulk_commit();
                 }
+                if (bo + lane < vw) yg[w0 + bo + lane] = so[bo + lane];
             } else {
                 __syncthreads();
                 stage_out_1d(yg, a.n_out, o0, s_out[k], kTileOut, kThreads);
