@@ -180,7 +180,8 @@ def build_cases(cfg_id, device, designs=(0, 1, 2), scale=None):
 
 
 def build_strided_cases(device):
-    """Stride-2 forms (Table 2, cell 6) at the sizes of configurations 2 and 5: OS and IS designs."""
+    """Stride-2 forms (Table 2, cell 6) at the sizes of configurations 2 and 5 (OS and IS designs), and separable
+    filters on the images of configuration 5."""
     import torch
     from paper_2010_15884_b200 import binding as B
     from paper_2010_15884_b200 import inputs
@@ -223,6 +224,18 @@ def build_strided_cases(device):
                               checked(B.sysconv2d_strided, x2.data_ptr(), wd, h, wd, h * wd, w, k, k, 2, 2,
                                       yd.data_ptr(), y_pitch, oh * y_pitch, batch, B.F32, d, stream),
                               n_out, x.size * 4 + 4 * n_out, n_out * k * k))
+    # separable filters (rank-one u v^T) on the same images: P + Q multiply-adds per output
+    for k in (3, 9, 15):
+        u = rng.normal(0, 1.0 / np.sqrt(k), k).astype(np.float32)
+        v = rng.normal(0, 1.0 / np.sqrt(k), k).astype(np.float32)
+        oh, ow = h - k + 1, wd - k + 1
+        y_pitch = (ow + 3) // 4 * 4
+        yd = torch.empty((batch, oh, y_pitch), dtype=torch.float32, device=device)
+        keep += [u, v, yd]
+        n_out = batch * oh * ow
+        cases.append(Case("5/separable", "%d+%d" % (k, k), B.OS,
+                          checked(B.sysconv2d_separable, x2.data_ptr(), wd, h, wd, h * wd, u, v, yd.data_ptr(), y_pitch,
+                                  oh * y_pitch, batch, stream), n_out, x.size * 4 + 4 * n_out, n_out * 2 * k))
     return cases, keep
 
 

@@ -136,6 +136,20 @@ int sysconv2d_strided(const void *x_dev, int width, int height, long long x_pitc
                       int dtype, int design, void *stream);
 
 /*
+ * Separable 2-D convolution, a second workload on the same folded array:
+ *   y[r][c] = sum_{i<p} sum_{k<q} u[i] * v[k] * x[r+i][c+k]
+ * i.e. sysconv2d with the rank-one filter w[i][k] = u[i]*v[k] (Gaussian blur, box, Sobel, ...), computed as one
+ * 1-D output-stationary (FBS) pass with the horizontal taps v per input row (Section 6's "multiple FBS 1-D
+ * convolutions") whose result feeds the p partial output rows through the vertical taps u: p + q
+ * multiply-adds per output instead of p * q.  The intermediate row is rounded to fp32 once.
+ *   u_host  HOST pointer to the p vertical taps (filter rows),  v_host  HOST pointer to the q horizontal taps
+ *   everything else as for sysconv2d; fp32 only, 1 <= p, q <= 15, batch <= 65535 (SYSCONV_EUNSUPPORTED beyond).
+ */
+int sysconv2d_separable(const void *x_dev, int width, int height, long long x_pitch, long long x_batch_stride,
+                        const void *u_host, int p, const void *v_host, int q,
+                        void *y_dev, long long y_pitch, long long y_batch_stride, int batch, void *stream);
+
+/*
  * Generic space-time-transform executor (Sections 2.1-2.2 and the generic code pattern of Section 4).
  * The 1-D convolution UREs over the iteration space (c, q) are mapped by PE = p_c*c + p_q*q and
  * time = s_c*c + s_q*q; the dependences, delays and PE distances are derived from (P, s) alone, so the six

@@ -13,7 +13,7 @@ seeded synthetic workloads.
 
 _BINDING_NAMES = (
     "sysconv1d", "sysconv2d", "sysconv1d_strided", "sysconv2d_strided", "sysconv1d_host", "sysconv2d_host",
-    "sysconv1d_host_static", "static_scratch_bytes", "conv1d", "conv2d", "spacetime_describe", "sysconv1d_spacetime", "sysconv1d_host_multi", "host_multi_workspace_bytes",
+    "sysconv1d_host_static", "static_scratch_bytes", "conv1d", "conv2d", "spacetime_describe", "sysconv1d_spacetime", "sysconv2d_separable", "conv2d_separable", "sysconv1d_host_multi", "host_multi_workspace_bytes",
     "load_library", "library_path", "SysconvError", "WS", "OS", "IS", "FSM", "BFS", "FFS", "F32", "U8S8_S32",
     "DESIGN_NAMES", "status_string", "design_name", "version", "host_workspace_bytes",
     "launch_count", "device_status",

@@ -54,6 +54,9 @@ def load_library():
     lib.sysconv2d_strided.restype = _c_int
     lib.sysconv2d_strided.argtypes = [_vp, _c_int, _c_int, _c_ll, _c_ll, _vp, _c_int, _c_int, _c_int, _c_int, _vp,
                                       _c_ll, _c_ll, _c_int, _c_int, _c_int, _vp]
+    lib.sysconv2d_separable.restype = _c_int
+    lib.sysconv2d_separable.argtypes = [_vp, _c_int, _c_int, _c_ll, _c_ll, _vp, _c_int, _vp, _c_int, _vp, _c_ll, _c_ll,
+                                        _c_int, _vp]
     lib.sysconv_spacetime_describe.restype = _c_int
     lib.sysconv_spacetime_describe.argtypes = [_c_int, _c_int, _c_int, _c_int, _c_int, _vp, _vp]
     lib.sysconv1d_spacetime.restype = _c_int
@@ -161,6 +164,38 @@ def sysconv2d_strided(x_ptr, width, height, x_pitch, x_batch_stride, w_host, q, 
     return int(lib.sysconv2d_strided(_vp(x_ptr), width, height, x_pitch, x_batch_stride,
                                      w_host.ctypes.data_as(_vp), q, p, stride_c, stride_r, _vp(y_ptr), y_pitch,
                                      y_batch_stride, batch, dtype, design, _vp(stream_ptr)))
+
+
+def sysconv2d_separable(x_ptr, width, height, x_pitch, x_batch_stride, u_host, v_host, y_ptr, y_pitch, y_batch_stride,
+                        batch, stream_ptr):
+    """Raw call: u_host = vertical taps (filter rows), v_host = horizontal taps, float32 numpy arrays."""
+    lib = load_library()
+    return int(lib.sysconv2d_separable(_vp(x_ptr), width, height, x_pitch, x_batch_stride,
+                                       u_host.ctypes.data_as(_vp), int(u_host.shape[0]), v_host.ctypes.data_as(_vp),
+                                       int(v_host.shape[0]), _vp(y_ptr), y_pitch, y_batch_stride, batch,
+                                       _vp(stream_ptr)))
+
+
+def conv2d_separable(x, u, v, out=None, stream=None):
+    """y[b, r, c] = sum_i sum_k u[i] v[k] x[b, r+i, c+k] on float32 CUDA tensors. x: (h, w) or (batch, h, w)."""
+    import torch
+    if not x.is_cuda:
+        raise SysconvError(-1, "conv2d_separable (x is not a CUDA tensor; there is no CPU path)")
+    squeeze = x.dim() == 2
+    x3 = x.unsqueeze(0) if squeeze else x
+    if x3.dim() != 3 or x3.stride(2) != 1 or x3.dtype != torch.float32:
+        raise ValueError("x must be float32, (h, w) or (batch, h, w) with contiguous rows")
+    u = np.ascontiguousarray(u, dtype=np.float32).reshape(-1)
+    v = np.ascontiguousarray(v, dtype=np.float32).reshape(-1)
+    batch, h, wd = x3.shape
+    if out is None:
+        out = torch.empty((batch, max(h - len(u) + 1, 0), max(wd - len(v) + 1, 0)), dtype=torch.float32, device=x.device)
+    y3 = out.unsqueeze(0) if out.dim() == 2 else out
+    st = sysconv2d_separable(x3.data_ptr(), wd, h, x3.stride(1), x3.stride(0) if batch > 1 else 0, u, v, y3.data_ptr(),
+                             y3.stride(1), y3.stride(0) if batch > 1 else 0, batch, _stream_ptr(stream))
+    if st != 0:
+        raise SysconvError(st, "sysconv2d_separable")
+    return out.squeeze(0) if (squeeze and out.dim() == 3) else out
 
 
 def spacetime_describe(P, s, q):

@@ -258,6 +258,35 @@ int sysconv2d_strided(const void *x_dev, int width, int height, long long x_pitc
     return finish(err, launches);
 }
 
+int sysconv2d_separable(const void *x_dev, int width, int height, long long x_pitch, long long x_batch_stride,
+                        const void *u_host, int p, const void *v_host, int q, void *y_dev, long long y_pitch,
+                        long long y_batch_stride, int batch, void *stream)
+{
+    using namespace sysconv;
+    if (!x_dev || !y_dev || !u_host || !v_host) return SYSCONV_EINVAL;
+    if (q < 1 || p < 1 || width < q || height < p || batch < 1) return SYSCONV_EINVAL;
+    const int out_w = width - q + 1, out_h = height - p + 1;
+    if (x_pitch < width || y_pitch < out_w) return SYSCONV_EINVAL;
+    const long long x_img = (long long)(height - 1) * x_pitch + width;
+    const long long y_img = (long long)(out_h - 1) * y_pitch + out_w;
+    if (batch > 1 && (x_batch_stride < x_img || y_batch_stride < y_img)) return SYSCONV_EINVAL;
+    if (batch == 1) { x_batch_stride = x_img; y_batch_stride = y_img; }
+    const unsigned long long x_bytes = ((unsigned long long)(batch - 1) * x_batch_stride + x_img) * 4ull;
+    const unsigned long long y_bytes = ((unsigned long long)(batch - 1) * y_batch_stride + y_img) * 4ull;
+    if (overlaps(x_dev, x_bytes, y_dev, y_bytes)) return SYSCONV_EINVAL;
+    if (q > kMaxQ2 || p > kMaxP2 || batch > 65535) return SYSCONV_EUNSUPPORTED;
+    Conv2DArgs a;
+    a.x = x_dev; a.y = y_dev;
+    a.width = width; a.height = height; a.out_w = out_w; a.out_h = out_h;
+    a.x_pitch = x_pitch; a.y_pitch = y_pitch;
+    a.x_bstride = x_batch_stride; a.y_bstride = y_batch_stride; a.batch = batch;
+    int launches = 0;
+    const cudaError_t err = launch_conv2d_f32_separable(a, static_cast<const float *>(u_host), p,
+                                                        static_cast<const float *>(v_host), q,
+                                                        static_cast<cudaStream_t>(stream), &launches);
+    return finish(err, launches);
+}
+
 int sysconv_spacetime_describe(int p_c, int p_q, int s_c, int s_q, int q, int *info, char *name)
 {
     return sysconv::spacetime_describe(p_c, p_q, s_c, s_q, q, info, name);

@@ -89,6 +89,10 @@ cudaError_t launch_conv1d_f32_stride2(int design, const Conv1DArgs &a, const flo
 cudaError_t launch_conv2d_f32_stride2(int design, const Conv2DArgs &a, const float *w, int q, int p, cudaStream_t s,
                                       int *launches);
 
+// separable 2-D convolution (conv2d_f32_sep.cu): u = p vertical taps, v = q horizontal taps
+cudaError_t launch_conv2d_f32_separable(const Conv2DArgs &a, const float *u, int p, const float *v, int q, cudaStream_t s,
+                                        int *launches);
+
 // generic space-time executor (spacetime.cu): *status receives the planning result
 int spacetime_describe(int pc, int pq, int sc, int sq, int q, int *out10, char *name4);
 cudaError_t launch_spacetime_conv1d(const float *x, long long n, const float *w, int q, float *y, int pc, int pq, int sc,

@@ -26,7 +26,7 @@ def _declared_functions():
 def test_header_declares_the_expected_entry_points():
     names = _declared_functions()
     for must in ("sysconv1d", "sysconv2d", "sysconv1d_strided", "sysconv2d_strided", "sysconv_spacetime_describe",
-                 "sysconv1d_spacetime", "sysconv1d_host", "sysconv1d_host_multi", "sysconv2d_host", "sysconv_status_string",
+                 "sysconv1d_spacetime", "sysconv2d_separable", "sysconv1d_host", "sysconv1d_host_multi", "sysconv2d_host", "sysconv_status_string",
                  "sysconv_design_name", "sysconv_version", "sysconv_launch_count"):
         assert must in names
 
@@ -120,3 +120,16 @@ def test_host_multi_argument_validation_needs_no_gpu(lib):
     assert call(vp(x.ctypes.data), 1000, 1, wp, q, d, yp, b.F32, vp(0x7f0000000000), 100, vp(0)) == 1       # workspace too small
     assert call(vp(x.ctypes.data), 1000, 1, wp, q, d, yp, b.F32, vp(0x7f0000000010), 1 << 20, vp(0)) == 1   # misaligned workspace
     assert call(vp(x.ctypes.data), 1000, 1, wp, q, d, yp, b.U8S8_S32, vp(0x7f0000000000), 1 << 20, vp(0)) == 2
+
+
+def test_separable_argument_validation_needs_no_gpu(lib):
+    import numpy as np
+    from paper_2010_15884_b200 import binding as b
+    u, v = np.ones(3, np.float32), np.ones(5, np.float32)
+    x, y = 0x10000, 0x90000000
+    assert b.sysconv2d_separable(0, 64, 64, 64, 0, u, v, y, 60, 0, 1, 0) == 1           # null x
+    assert b.sysconv2d_separable(x, 4, 64, 4, 0, u, v, y, 1, 0, 1, 0) == 1              # image narrower than v
+    assert b.sysconv2d_separable(x, 64, 64, 64, 0, u, v, y, 59, 0, 1, 0) == 1           # y_pitch < out_w
+    assert b.sysconv2d_separable(x, 64, 64, 64, 0, u, v, y, 60, 0, 0, 0) == 1           # batch < 1
+    assert b.sysconv2d_separable(x, 64, 64, 64, 0, np.ones(16, np.float32), v, y, 60, 0, 1, 0) == 2   # 16 vertical taps
+    assert b.sysconv2d_separable(x, 64, 64, 64, 64 * 64, u, v, y, 60, 62 * 60, 70000, 0) == 2         # batch beyond 65535

@@ -561,6 +561,84 @@ def test_2d_stride2_full_hd_sampled(cuda_device):
         assert_close_f32(y.cpu().numpy()[0][rows, cols], y_ref, s_ref, "sampled, %s" % B.DESIGN_NAMES[design])
 
 
+# ------------------------------------------------------------------------ separable 2-D convolution
+
+
+def check_separable(x_np, u, v, device, x_pitch=None, y_pitch=None, x_off=0, y_off=0):
+    batch, h, wd = x_np.shape
+    p, q = len(u), len(v)
+    oh, ow = h - p + 1, wd - q + 1
+    x_pitch = x_pitch or wd
+    y_pitch = y_pitch or ow
+    xb = torch.zeros(x_off + batch * h * x_pitch + 16, dtype=torch.float32, device=device)
+    yb = torch.full((y_off + batch * oh * y_pitch + 64,), CANARY, dtype=torch.float32, device=device)
+    xb[x_off: x_off + batch * h * x_pitch].view(batch, h, x_pitch)[:, :, :wd] = torch.from_numpy(x_np).to(device)
+    st = B.sysconv2d_separable(xb.data_ptr() + 4 * x_off, wd, h, x_pitch, h * x_pitch, u, v, yb.data_ptr() + 4 * y_off,
+                               y_pitch, oh * y_pitch, batch, torch.cuda.current_stream().cuda_stream)
+    assert st == 0, B.status_string(st)
+    torch.cuda.synchronize()
+    yh = yb.cpu().numpy()
+    body = yh[y_off: y_off + batch * oh * y_pitch].reshape(batch, oh, y_pitch)
+    assert (body[:, :, ow:] == CANARY).all(), "write into the pitch padding"
+    assert (yh[:y_off] == CANARY).all() and (yh[y_off + batch * oh * y_pitch:] == CANARY).all()
+    w = np.outer(u.astype(np.float64), v.astype(np.float64)).astype(np.float32)
+    for b in range(batch):
+        # the definition: Eq. 3 with the rank-one filter u v^T (fp32 product of the taps, as the oracle takes fp32 taps)
+        y_ref, s_ref = oracle.conv2d_f32(x_np[b], w)
+        assert_close_f32(body[b, :, :ow], y_ref, 1.0001 * s_ref + 1e-30, "image %d" % b)
+
+
+@pytest.mark.parametrize("pq", [(1, 1), (3, 3), (5, 5), (7, 7), (8, 8), (9, 9), (15, 15), (2, 11), (13, 4), (15, 1), (1, 15),
+                                (7, 15), (8, 3)], ids=lambda f: "%dx%d" % f)
+def test_separable_filter_shapes(cuda_device, pq):
+    p, q = pq
+    rng = np.random.default_rng(1000 + 16 * p + q)
+    x = rng.random((2, 75, 700), dtype=np.float32)
+    u = rng.uniform(-1, 1, p).astype(np.float32)
+    v = rng.uniform(-1, 1, q).astype(np.float32)
+    check_separable(x, u, v, cuda_device)
+    check_separable(x[:, :, :301], u, v, cuda_device, x_pitch=307, y_pitch=303, x_off=1, y_off=1)
+
+
+@pytest.mark.parametrize("hw", [(0, 0), (1, 0), (0, 1), (2, 3), (31, 127), (32, 128), (33, 129), (40, 255), (7, 513), (70, 1030)])
+@pytest.mark.parametrize("pq", [(3, 3), (5, 7), (15, 15)], ids=lambda f: "%dx%d" % f)
+def test_separable_ragged_image_sizes(cuda_device, pq, hw):
+    p, q = pq
+    rng = np.random.default_rng(1100 + hw[0] + hw[1])
+    x = rng.random((1, p + hw[0], q + hw[1]), dtype=np.float32)
+    check_separable(x, rng.uniform(-1, 1, p).astype(np.float32), rng.uniform(-1, 1, q).astype(np.float32), cuda_device)
+
+
+def test_separable_exact_on_integers_and_equal_to_the_full_convolution(cuda_device):
+    # integer-valued data and taps: every order of summation is exact, so the separable result must equal the
+    # full 2-D convolution with the outer-product filter bit for bit
+    rng = np.random.default_rng(7)
+    x = rng.integers(-8, 9, (2, 300, 1200)).astype(np.float32)
+    u = rng.integers(-3, 4, 5).astype(np.float32)
+    v = rng.integers(-3, 4, 9).astype(np.float32)
+    xd = torch.from_numpy(x).to(cuda_device)
+    y = B.conv2d_separable(xd, u, v)
+    full = B.conv2d(xd, np.outer(u, v).astype(np.float32), B.OS)
+    torch.cuda.synchronize()
+    assert torch.equal(y, full)
+    ref, _ = oracle.conv2d_f32(x[1], np.outer(u, v).astype(np.float32))
+    np.testing.assert_array_equal(y[1].cpu().numpy().astype(np.float64), ref)
+
+
+def test_separable_full_size_sampled(cuda_device):
+    x, _ = inputs.make_config(5, dict(filters=[3], batch=2))
+    rng = np.random.default_rng(8)
+    u = rng.normal(0, 1 / 3, 9).astype(np.float32)
+    v = rng.normal(0, 1 / 3, 9).astype(np.float32)
+    y = B.conv2d_separable(torch.from_numpy(x).to(cuda_device), u, v)
+    torch.cuda.synchronize()
+    oh, ow = 4096 - 8, 4096 - 8
+    rows = np.concatenate([rng.integers(0, oh, 3000), [0, 0, oh - 1, oh - 1]])
+    cols = np.concatenate([rng.integers(0, ow, 3000), [0, ow - 1, 0, ow - 1]])
+    y_ref, s_ref = oracle.conv2d_f32_at(x[1], np.outer(u.astype(np.float64), v.astype(np.float64)).astype(np.float32), rows, cols)
+    assert_close_f32(y[1].cpu().numpy()[rows, cols], y_ref, 1.0001 * s_ref + 1e-30, "sampled")
+
+
 # ------------------------------------------------------------------------ generic space-time executor
 
 ST_PAPER = {"SBM": ((1, 1), (0, 1)), "BSM": ((0, 1), (1, 1)), "FSM": ((0, 1), (1, -1)), "BFS": ((1, 0), (1, 1)),
