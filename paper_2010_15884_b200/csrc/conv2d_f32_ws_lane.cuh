@@ -4,7 +4,7 @@
 // An array has only Q <= 15 PEs, so it lives entirely in one lane (PE-to-PE transfer = register renaming, no
 // shuffle); all arrays hold the same filter, so the stationary taps are uniform operands from the kernel
 // parameters.  A CTA is one warp = 32 arrays stacked over 128 output rows (array a: rows 4a .. 4a+3, which
-// share the broadcast inputs); it streams a segment of the image width, eight image columns at a time.
+// share the broadcast inputs); it streams a segment of the image width, 8 (small filters: 16) image columns at a time.
 //
 // Macro-step T broadcasts the P+3 inputs x(4a .. 4a+P+2, T) of image column T to the array.  The sums of two
 // neighbouring outputs o (even) and o+1 of a row travel together in one 64-bit register pair, which sits in
@@ -14,12 +14,12 @@
 // pair leaves PE Q-1 with its second sum one filter column short, which the emission adds with P scalar
 // FMAs: no zero tap ever multiplies an input.
 //
-// Data movement: the chunk of 8 image columns x 142 rows is loaded with 128-bit loads (one 32-byte sector per
-// row), held in registers while the previous chunk is processed, and written TRANSPOSED ([column][row]) to
+// Data movement: the chunk of 8 (16) image columns x 142 rows is loaded with 128-bit loads (one or two 32-byte
+// sectors per row), held in registers while the previous chunk is processed, and written TRANSPOSED ([column][row]) to
 // shared memory, so that an array reads its inputs of one image column with 128-bit loads that are contiguous
 // across the lanes.  Outputs go the other way: the four rows' results of one column leave as one 128-bit
-// store into a transposed ring of 16 or 32 columns, and complete groups of 8 columns are written to memory as
-// full 32-byte sectors per row.
+// store into a transposed ring of 16 or 32 columns, and complete groups of 8 (16) columns are written to memory
+// as full 32-byte sectors per row.
 #pragma once
 
 #include "conv2d_f32_is_pair.cuh"
@@ -28,8 +28,15 @@ namespace sysconv {
 
 constexpr int kWlM = 4;                         // output rows per array
 constexpr int kWlRows = kLanes * kWlM;          // 128 output rows per CTA (one warp)
-constexpr int kWlChunk = 8;                     // image columns per staged chunk
+// Image columns per staged chunk.  Small filters are bound by the load/store unit: a warp's 128-bit global
+// access covers 16 rows (16 cache lines) with 8-column chunks, 8 rows with 16-column chunks, so the wider chunk
+// halves the work of the memory pipe per byte; larger filters keep the narrow chunk (registers, shared memory).
+template <int P, int Q>
+struct WlShape {
+    static constexpr int kChunk = P * Q <= 25 ? 16 : 8;
+};
 constexpr int kWlPitch = 164;                   // rows per staged column: >= 128 + 14, = 4 mod 32 (conflict-free transposes)
+constexpr int kWlPitchO = 132;                  // rows per column of the output ring: >= 128, = 4 mod 32
 
 template <int P, int Q>
 __global__ void __launch_bounds__(kLanes)
@@ -41,11 +48,14 @@ conv2d_ws_lane_kernel(const Conv2DArgs a, const __grid_constant__ Taps2D taps, c
     constexpr int K = M + P - 1;                // input rows feeding M output rows
     constexpr int KG = (K + 3) / 4;
     constexpr int kRowsUsed = kWlRows + P - 1;  // staged rows that are ever read (the last group may read up to 3 more)
-    constexpr int kGroupDelay = (Q - 1 + 7) / 8;    // chunks between an output group's first input and its completion
-    constexpr int kWlRing = kGroupDelay <= 1 ? 16 : 32;     // columns of the output ring: groups j-delay .. j are alive
+    constexpr int kWlChunk = WlShape<P, Q>::kChunk;
+    constexpr int WPR = kWlChunk / 4;           // 128-bit words per row of a chunk
+    constexpr int kGroupDelay = (Q - 1 + kWlChunk - 1) / kWlChunk;  // chunks between an output group's first input and its completion
+    // columns of the output ring: groups j-delay .. j are alive (a power of two)
+    constexpr int kWlRing = (kGroupDelay + 1) * kWlChunk <= 16 ? 16 : ((kGroupDelay + 1) * kWlChunk <= 32 ? 32 : 64);
     static_assert(kWlRows + 4 * KG - M <= kWlPitch, "staged column too short");
     __shared__ __align__(16) float s_x[kWlChunk * kWlPitch];
-    __shared__ __align__(16) float s_o[kWlRing * kWlPitch];
+    __shared__ __align__(16) float s_o[kWlRing * kWlPitchO];
 
     const int lane = threadIdx.x;
     const int band0 = blockIdx.y * kWlRows;             // first output row of the CTA
@@ -56,15 +66,16 @@ conv2d_ws_lane_kernel(const Conv2DArgs a, const __grid_constant__ Taps2D taps, c
     const bool x_vec = row_alignment(static_cast<const float *>(a.x), a.x_pitch, a.x_bstride, a.batch) == 4;
     const int y_align = row_alignment(static_cast<const float *>(a.y), a.y_pitch, a.y_bstride, a.batch);
 
-    // staging of image columns [cc, cc+8) x rows [band0, band0 + kRowsUsed): two 128-bit words per row
-    constexpr int kStageVec = (kRowsUsed * 2 + kLanes - 1) / kLanes;
+    // staging of image columns [cc, cc+chunk) x rows [band0, band0 + kRowsUsed): WPR 128-bit words per row
+    // (a permutation that makes the transposed stores of the four-word case conflict-free was measured: no gain)
+    constexpr int kStageVec = (kRowsUsed * WPR + kLanes - 1) / kLanes;
     float pf[kStageVec][4];
     auto stage_load = [&](int cc) {
 #pragma unroll
         for (int n = 0; n < kStageVec; ++n) {
             const int idx = lane + n * kLanes;
-            const int row = idx >> 1, i = idx & 1;
-            if (idx < kRowsUsed * 2) {
+            const int row = idx / WPR, i = idx % WPR;
+            if (idx < kRowsUsed * WPR) {
                 const float *rowp = xb + static_cast<long long>(min(band0 + row, a.height - 1)) * a.x_pitch;
                 load_group<Tr>(rowp, cc + 4 * i, a.width, x_vec, pf[n]);
             }
@@ -74,23 +85,23 @@ conv2d_ws_lane_kernel(const Conv2DArgs a, const __grid_constant__ Taps2D taps, c
 #pragma unroll
         for (int n = 0; n < kStageVec; ++n) {
             const int idx = lane + n * kLanes;
-            const int row = idx >> 1, i = idx & 1;
-            if (idx < kRowsUsed * 2) {
+            const int row = idx / WPR, i = idx % WPR;
+            if (idx < kRowsUsed * WPR) {
 #pragma unroll
                 for (int e = 0; e < 4; ++e) s_x[(4 * i + e) * kWlPitch + row] = pf[n][e];
             }
         }
     };
-    // write output columns [c0 + 8g, c0 + 8g + 8) of the CTA's 128 rows from the ring to memory
+    // write output columns [c0 + chunk*g, c0 + chunk*(g+1)) of the CTA's 128 rows from the ring to memory
     auto flush = [&](int g) {
-        const int ocol = c0 + 8 * g;
+        const int ocol = c0 + kWlChunk * g;
 #pragma unroll
-        for (int n = 0; n < kWlRows * 2 / kLanes; ++n) {
+        for (int n = 0; n < kWlRows * WPR / kLanes; ++n) {
             const int idx = lane + n * kLanes;
-            const int row = idx >> 1, i = idx & 1;
+            const int row = idx / WPR, i = idx % WPR;
             float v[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) v[e] = s_o[((8 * g + 4 * i + e) & (kWlRing - 1)) * kWlPitch + row];
+            for (int e = 0; e < 4; ++e) v[e] = s_o[((kWlChunk * g + 4 * i + e) & (kWlRing - 1)) * kWlPitchO + row];
             if (band0 + row < a.out_h)
                 store_group<Tr>(yb + static_cast<long long>(band0 + row) * a.y_pitch, ocol + 4 * i, c1, y_align, v);
         }
@@ -107,9 +118,9 @@ conv2d_ws_lane_kernel(const Conv2DArgs a, const __grid_constant__ Taps2D taps, c
     stage_store();
     __syncwarp();
 #pragma unroll 1
-    for (int j = 0; (j - kGroupDelay) * 8 < n_out; ++j) {
+    for (int j = 0; (j - kGroupDelay) * kWlChunk < n_out; ++j) {
         stage_load(c0 + (j + 1) * kWlChunk);
-        // small filters: all eight macro-steps of the chunk unrolled (immediate shared-memory offsets, the reads
+        // small filters: all macro-steps of the chunk unrolled (immediate shared-memory offsets, the reads
         // of later columns can be issued early); larger ones: two macro-steps per iteration (code size)
         constexpr int kUnrollU = P * Q <= 25 ? kWlChunk / 2 : 1;
 #pragma unroll kUnrollU
@@ -135,9 +146,9 @@ conv2d_ws_lane_kernel(const Conv2DArgs a, const __grid_constant__ Taps2D taps, c
                         e1[m] = z;
                     }
                     const int o = j * kWlChunk + c - Q;     // may be negative during the fill: those slots are rewritten
-                    *reinterpret_cast<float4 *>(s_o + (o & (kWlRing - 1)) * kWlPitch + 4 * lane) =
+                    *reinterpret_cast<float4 *>(s_o + (o & (kWlRing - 1)) * kWlPitchO + 4 * lane) =
                         make_float4(e0[0], e0[1], e0[2], e0[3]);
-                    *reinterpret_cast<float4 *>(s_o + ((o + 1) & (kWlRing - 1)) * kWlPitch + 4 * lane) =
+                    *reinterpret_cast<float4 *>(s_o + ((o + 1) & (kWlRing - 1)) * kWlPitchO + 4 * lane) =
                         make_float4(e1[0], e1[1], e1[2], e1[3]);
                 }
 #pragma unroll
@@ -183,7 +194,8 @@ cudaError_t launch_conv2d_ws_lane(const Conv2DArgs &a, const Taps2D &taps, cudaS
     if (segs > max_segs) segs = max_segs;
     if (segs < 1) segs = 1;
     int seg_w = static_cast<int>((a.out_w + segs - 1) / segs);
-    seg_w = (seg_w + kWlChunk - 1) / kWlChunk * kWlChunk;
+    constexpr int kChunk = WlShape<P, Q>::kChunk;
+    seg_w = (seg_w + kChunk - 1) / kChunk * kChunk;
     dim3 grid((a.out_w + seg_w - 1) / seg_w, static_cast<unsigned>(bands), a.batch);
     if (grid.y > 65535) return cudaErrorInvalidConfiguration;
     conv2d_ws_lane_kernel<P, Q><<<grid, kLanes, 0, s>>>(a, taps, tp, seg_w);
