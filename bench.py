@@ -498,14 +498,14 @@ def run_ours(args):
 # here because traffic grows in proportion to the number of images) and profiles/conv2d_u8_cfg4_kernels.md (full
 # size; the 33 MB of outputs stay dirty in L2 past the end of the kernel, so only the reads show).
 NCU_TRAFFIC = {
-    "cfg2 WS Q=4": 482395648, "cfg2 OS Q=4": 482511616, "cfg2 IS Q=4": 481227520,
-    "cfg2 WS Q=16": 482588672, "cfg2 OS Q=16": 483188480, "cfg2 IS Q=16": 482079488,
-    "cfg2 WS Q=32": 486472192, "cfg2 OS Q=32": 489061632, "cfg2 IS Q=32": 487247104,
-    "cfg5 WS 3x3": 8 * 265239296, "cfg5 OS 3x3": 8 * 223642368, "cfg5 IS 3x3": 8 * 224715264,
-    "cfg5 WS 9x9": 8 * 271866368, "cfg5 OS 9x9": 8 * 235974656, "cfg5 IS 9x9": 8 * 236198656,
-    "cfg5 WS 15x15": 8 * 282769408, "cfg5 OS 15x15": 8 * 239437824, "cfg5 IS 15x15": 8 * 240289792,
-    "cfg4 WS 3x3": 11126784, "cfg4 OS 3x3": 8303872, "cfg4 IS 3x3": 8306176,
-    "cfg4 WS 7x7": 10518272, "cfg4 OS 7x7": 8307456, "cfg4 IS 7x7": 8316928,
+    "cfg2 WS Q=4": 481693184, "cfg2 OS Q=4": 481795328, "cfg2 IS Q=4": 481168128,
+    "cfg2 WS Q=16": 481935616, "cfg2 OS Q=16": 482634240, "cfg2 IS Q=16": 482909696,
+    "cfg2 WS Q=32": 487177728, "cfg2 OS Q=32": 489519360, "cfg2 IS Q=32": 488174336,
+    "cfg5 WS 3x3": 8 * 255084544, "cfg5 OS 3x3": 8 * 223725312, "cfg5 IS 3x3": 8 * 225803776,
+    "cfg5 WS 9x9": 8 * 271382272, "cfg5 OS 9x9": 8 * 236015616, "cfg5 IS 9x9": 8 * 236046848,
+    "cfg5 WS 15x15": 8 * 290182400, "cfg5 OS 15x15": 8 * 238945280, "cfg5 IS 15x15": 8 * 241408256,
+    "cfg4 WS 3x3": 10991104, "cfg4 OS 3x3": 8311552, "cfg4 IS 3x3": 8306944,
+    "cfg4 WS 7x7": 10485248, "cfg4 OS 7x7": 8311040, "cfg4 IS 7x7": 8315136,
 }
 
 
