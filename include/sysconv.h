@@ -261,11 +261,22 @@ const char *sysconv_design_name(int design);
  * Device-side health check.  The pipelined kernels wait for their asynchronous
  * copies with a bounded number of polls; a kernel whose limit runs out stops
  * taking work, raises a flag in device memory and returns normally (its outputs
- * are then incomplete).  This call synchronises the current device with a
- * blocking copy, returns SYSCONV_ETIMEOUT if the flag was raised since the last
- * call (and clears it), SYSCONV_OK otherwise.
+ * are then incomplete).  This call synchronises the current device (every
+ * stream, cudaDeviceSynchronize), returns SYSCONV_ETIMEOUT if the flag was
+ * raised since the last call (and clears it), SYSCONV_OK otherwise.
  */
 int sysconv_device_status(void);
+
+/*
+ * Self-test of that mechanism (no counterpart in the paper; for the test suite).
+ * Enqueues one small block on `stream` that arms a shared-memory barrier for
+ * bytes which are never sent -- it issues no copy, so nothing is in flight
+ * towards it -- polls 1024 times, gives up the way the pipelined kernels do
+ * (raises the flag, returns normally) and ends.  The next
+ * sysconv_device_status() must return SYSCONV_ETIMEOUT, the one after it
+ * SYSCONV_OK.  Touches no caller memory.
+ */
+int sysconv_selftest_wait_timeout(void *stream);
 
 /* Library version, major*10000 + minor*100 + patch. */
 int sysconv_version(void);

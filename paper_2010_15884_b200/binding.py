@@ -83,6 +83,8 @@ def load_library():
     lib.sysconv_design_name.argtypes = [_c_int]
     lib.sysconv_version.restype = _c_int
     lib.sysconv_device_status.restype = _c_int
+    lib.sysconv_selftest_wait_timeout.restype = _c_int
+    lib.sysconv_selftest_wait_timeout.argtypes = [_vp]
     lib.sysconv_launch_count.restype = _c_ll
     _lib = lib
     return lib
@@ -105,6 +107,13 @@ def version():
 def device_status():
     """0 if no kernel gave up a bounded wait on the current device since the last call, else 4 (time-out)."""
     return int(load_library().sysconv_device_status())
+
+
+def selftest_wait_timeout(stream=None):
+    """Enqueue the one-block self-test whose bounded wait runs out; the next device_status() reports 4."""
+    st = int(load_library().sysconv_selftest_wait_timeout(_vp(_stream_ptr(stream))))
+    if st != 0:
+        raise SysconvError(st, "sysconv_selftest_wait_timeout")
 
 
 def launch_count():

@@ -414,10 +414,12 @@ conv1d_f32_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, const
         for (int k = 0; k < K; ++k) mbar_init(&full[k], 1);
         mbar_init_fence();
     }
-    // elements of tile k that arrive by bulk copy: the part of the tile inside the signal, in whole 16-byte words
+    // elements of tile k that arrive by bulk copy: the part of the tile inside the signal, in whole 16-byte words.
+    // A tile without outputs gets no copy at all: the issuing thread and the consumers use this one predicate,
+    // so no copy is ever issued that nobody waits for.
     auto bulk_in = [&](int k) -> int {
         const long long t0 = base + k * G::kTileOut;
-        if (!x_ok || t0 >= a.n) return 0;
+        if (!x_ok || t0 >= a.n_out) return 0;
         const long long valid = a.n - t0 < G::kTileIn ? a.n - t0 : G::kTileIn;
         return static_cast<int>(valid) & ~3;
     };
@@ -443,15 +445,15 @@ conv1d_f32_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, const
             if (t0 >= a.n_out) break;
             const int be = bulk_in(k);
             if (be > 0) {
-                const bool ok = mbar_wait_bounded(&full[k], phase);
+                const bool ok = mbar_wait_bounded(&full[k], phase, kWaitPolls);
                 const bool give_up = WARPS == 1 ? __any_sync(kFullMask, !ok) != 0 : __syncthreads_or(!ok) != 0;
                 if (give_up) {
                     if (threadIdx.x == 0) {
                         atomicExch(status_word, 1u);
-                        for (int j = k + 1; j < K; ++j)      // copies still in flight target this CTA's memory
-                            if (bulk_in(j) > 0) mbar_wait_bounded(&full[j], phase, 1u << 16);
-                        bulk_wait_read<0>();
+                        for (int j = k; j < K; ++j)          // copies still in flight target this CTA's memory
+                            if (bulk_in(j) > 0) mbar_wait_bounded(&full[j], phase, kGiveUpPolls);
                     }
+                    if (lane == 0) bulk_wait_read<0>();      // every warp's own bulk stores have read their source
                     return;
                 }
             }

@@ -1,9 +1,11 @@
 // C ABI of libsysconv.so: argument validation and dispatch.  See include/sysconv.h
 // for the contract of every entry point.  No device memory is allocated here.
 #include <atomic>
+#include <climits>
 #include <mutex>
 
 #include "sysconv_common.cuh"
+#include "tma_utils.cuh"
 
 // Raised (set to 1) by a kernel that gave up a bounded wait; read and cleared by sysconv_device_status().
 static __device__ unsigned g_status_word;
@@ -40,6 +42,34 @@ const DeviceInfo *device_info()
 
 inline size_t in_elt_bytes(int dtype) { return dtype == SYSCONV_F32 ? 4 : 1; }
 inline long long align256(long long v) { return (v + 255) & ~255LL; }
+
+// a * b * c for positive factors, or -1 if the product (plus alignment slack) would not fit a long long
+long long checked_product(long long a, long long b, long long c)
+{
+    const long long limit = LLONG_MAX / 4 - 256;
+    if (a <= 0 || b <= 0 || c <= 0) return -1;
+    if (a > limit / b) return -1;
+    const long long ab = a * b;
+    if (ab > limit / c) return -1;
+    return ab * c;
+}
+
+// One CTA that waits, bounded, for bytes nobody sends: it arms a shared-memory barrier with an expected
+// byte count, issues NO copy (so nothing is in flight towards the CTA), polls `polls` times, raises the
+// status word exactly as the pipelined kernels do when their limit runs out, and returns.
+__global__ void wait_timeout_selftest_kernel(unsigned *status_word, unsigned polls)
+{
+    __shared__ __align__(8) uint64_t bar;
+    if (threadIdx.x == 0) {
+        sysconv::mbar_init(&bar, 1);
+        sysconv::mbar_init_fence();
+        sysconv::mbar_arrive_expect_tx(&bar, 16);
+    }
+    __syncthreads();
+    const bool ok = sysconv::mbar_wait_bounded(&bar, 0, polls);
+    const bool give_up = __syncthreads_or(!ok) != 0;
+    if (give_up && threadIdx.x == 0) atomicExch(status_word, 1u);
+}
 
 int finish(cudaError_t err, int launches)
 {
@@ -344,15 +374,19 @@ long long sysconv1d_host_workspace_bytes(long long n, int q, int batch, int dtyp
 {
     if (q < 1 || n < q || batch < 1) return -1;
     if (dtype != SYSCONV_F32 && dtype != SYSCONV_U8S8_S32) return -1;
-    return align256(n * batch * (long long)in_elt_bytes(dtype)) + align256((n - q + 1) * batch * 4LL);
+    const long long in = checked_product(n, batch, (long long)in_elt_bytes(dtype));
+    const long long out = checked_product(n - q + 1, batch, 4LL);
+    if (in < 0 || out < 0) return -1;                    // sizes beyond the index type
+    return align256(in) + align256(out);
 }
 
 long long sysconv2d_host_workspace_bytes(int width, int height, int q, int p, int batch, int dtype)
 {
     if (q < 1 || p < 1 || width < q || height < p || batch < 1) return -1;
     if (dtype != SYSCONV_F32 && dtype != SYSCONV_U8S8_S32) return -1;
-    const long long in = (long long)width * height * batch * (long long)in_elt_bytes(dtype);
-    const long long out = (long long)(width - q + 1) * (height - p + 1) * batch * 4LL;
+    const long long in = checked_product((long long)width * height, batch, (long long)in_elt_bytes(dtype));
+    const long long out = checked_product((long long)(width - q + 1) * (height - p + 1), batch, 4LL);
+    if (in < 0 || out < 0) return -1;                    // sizes beyond the index type
     return align256(in) + align256(out);
 }
 
@@ -425,6 +459,7 @@ int sysconv1d_host(const void *x_host, long long n, const void *w_host, int q, v
 long long sysconv1d_host_multi_workspace_bytes(long long n, const int *q, int count, int dtype)
 {
     if (!q || count < 1 || count > 64 || dtype != SYSCONV_F32) return -1;
+    if (n < 1 || n > (LLONG_MAX / 4 - 256) / (4LL * (count + 1))) return -1;
     long long total = align256(n * 4LL);
     for (int j = 0; j < count; ++j) {
         if (q[j] < 1 || n < q[j]) return -1;
@@ -596,6 +631,8 @@ int sysconv_device_status(void)
     const DeviceInfo *d = device_info();
     if (!d) return SYSCONV_ECUDA;
     unsigned flag = 0;
+    // every stream of the device, non-blocking ones included: a kernel still running could raise the flag later
+    if (cudaDeviceSynchronize() != cudaSuccess) return SYSCONV_ECUDA;
     if (cudaMemcpy(&flag, d->status_word, sizeof(flag), cudaMemcpyDeviceToHost) != cudaSuccess) return SYSCONV_ECUDA;
     if (flag == 0) return SYSCONV_OK;
     flag = 0;
@@ -603,7 +640,15 @@ int sysconv_device_status(void)
     return SYSCONV_ETIMEOUT;
 }
 
-int sysconv_version(void) { return 101; }
+int sysconv_selftest_wait_timeout(void *stream)
+{
+    const DeviceInfo *d = device_info();
+    if (!d) return SYSCONV_ECUDA;
+    wait_timeout_selftest_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(d->status_word, 1u << 10);
+    return finish(cudaGetLastError(), 1);
+}
+
+int sysconv_version(void) { return 200; }
 
 long long sysconv_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

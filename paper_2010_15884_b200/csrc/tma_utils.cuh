@@ -1,7 +1,7 @@
 // Thin wrappers over the sm_100a asynchronous-copy PTX used by the pipelined kernels:
-// mbarrier objects in shared memory, bulk (TMA) copies global <-> shared, tiled tensor copies,
-// and the proxy fence that orders a thread's shared-memory writes before a bulk store.
-// No cluster multicast anywhere; every copy targets this GPU's own memory.
+// mbarrier objects in shared memory, bulk (TMA) copies global <-> shared, and the proxy fence
+// that orders a thread's shared-memory writes before a bulk store.
+// Every copy is issued by one CTA for itself and moves data of this GPU's own memory.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -44,9 +44,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
     return ok != 0;
 }
 
+// Poll limits of the bounded waits: a tile's copy gets kWaitPolls polls; once a CTA has given up, each of
+// its other copies gets kGiveUpPolls more before the CTA returns.
+constexpr uint32_t kWaitPolls = 1u << 22;
+constexpr uint32_t kGiveUpPolls = 1u << 16;
+
 // Wait for the phase with the given parity to complete, at most `limit` polls.
 // Returns false if the limit ran out (the caller records the time-out and leaves).
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, uint32_t limit = (1u << 22))
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t *bar, uint32_t parity, uint32_t limit = kWaitPolls)
 {
     for (uint32_t it = 0; it < limit; ++it)
         if (mbar_try_wait(bar, parity)) return true;
@@ -82,22 +87,5 @@ __device__ __forceinline__ void bulk_wait_read()
 
 // order this thread's generic-proxy shared-memory writes before later asynchronous-proxy reads
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-// 2-D tiled tensor copies (tensor map in kernel parameter space); c0 = innermost coordinate
-__device__ __forceinline__ void tensor_load_2d(void *smem_dst, const void *tmap, int c0, int c1, uint64_t *bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::
-            "r"(smem_u32(smem_dst)),
-        "l"(tmap), "r"(c0), "r"(c1), "r"(smem_u32(bar))
-        : "memory");
-}
-
-__device__ __forceinline__ void tensor_store_2d(const void *tmap, int c0, int c1, const void *smem_src)
-{
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%1, %2}], [%3];" ::"l"(tmap),
-                 "r"(c0), "r"(c1), "r"(smem_u32(smem_src))
-                 : "memory");
-}
 
 }  // namespace sysconv

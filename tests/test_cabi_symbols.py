@@ -133,3 +133,22 @@ def test_separable_argument_validation_needs_no_gpu(lib):
     assert b.sysconv2d_separable(x, 64, 64, 64, 0, u, v, y, 60, 0, 0, 0) == 1           # batch < 1
     assert b.sysconv2d_separable(x, 64, 64, 64, 0, np.ones(16, np.float32), v, y, 60, 0, 1, 0) == 2   # 16 vertical taps
     assert b.sysconv2d_separable(x, 64, 64, 64, 64 * 64, u, v, y, 60, 62 * 60, 70000, 0) == 2         # batch beyond 65535
+
+
+def test_size_queries_reject_products_beyond_the_index_type(lib):
+    # n * batch * 4 would wrap a signed 64-bit product to a small positive number: the queries must say -1 and the
+    # entry point that allocates nothing must answer "invalid argument" before anything is enqueued
+    import numpy as np
+    from paper_2010_15884_b200 import binding as b
+    n = (1 << 60) + 1024
+    assert lib.sysconv1d_host_workspace_bytes(ctypes.c_longlong(n), 4, 4, b.F32) == -1
+    assert lib.sysconv1d_host_workspace_bytes(ctypes.c_longlong(1 << 62), 4, 1, b.F32) == -1
+    assert lib.sysconv2d_host_workspace_bytes(1 << 30, 1 << 30, 3, 3, 1 << 20, b.F32) == -1
+    assert b.host_multi_workspace_bytes(1 << 61, [4, 16]) == -1
+    w = np.ones(4, np.float32)
+    before = b.launch_count()
+    vp = ctypes.c_void_p
+    st = lib.sysconv1d_host_static(vp(0x10000), ctypes.c_longlong(n), vp(w.ctypes.data), 4, vp(0x90000000), 4, b.F32, b.OS,
+                                   vp(0))
+    assert st == 1
+    assert b.launch_count() == before

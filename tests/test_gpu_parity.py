@@ -14,6 +14,7 @@ from paper_2010_15884_b200 import inputs
 pytestmark = pytest.mark.gpu
 
 DESIGNS = [B.WS, B.OS, B.IS]
+STRIDED_1D = [B.OS, B.IS]
 OTHER_DESIGNS = [B.FSM, B.BFS, B.FFS]        # the paper's other three 1-D designs (1-D fp32 only)
 TOL = 1e-5
 CANARY = 12345.0
@@ -125,6 +126,47 @@ def test_1d_many_tiles_sizes(cuda_device, design, q, n_out):
     x, ws = inputs.gen_1d_f32(n, [q], seed=2000 + q)
     y_ref, s_ref = oracle.conv1d_f32(x, ws[q])
     assert_close_f32(run_1d(x, ws[q], design, cuda_device), y_ref, s_ref, "n_out=%d q=%d" % (n_out, q))
+    assert B.device_status() == 0
+
+
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+@pytest.mark.parametrize("q", [5, 8, 17, 32])
+@pytest.mark.parametrize("tiles", [1, 2, 3, 4, 5, 8])
+def test_1d_output_count_a_whole_number_of_tiles(cuda_device, design, q, tiles):
+    """n_out an exact multiple of the 1216-output tile: the tile after the last one has no outputs, yet the signal's
+    last q-1 inputs lie in it.  One signal, and a batch (a block then walks on to the next signal)."""
+    n_out = 1216 * tiles
+    n = n_out + q - 1
+    x, ws = inputs.gen_1d_f32(n, [q], seed=2500 + q + tiles)
+    y_ref, s_ref = oracle.conv1d_f32(x, ws[q])
+    assert_close_f32(run_1d(x, ws[q], design, cuda_device), y_ref, s_ref, "n_out=%d q=%d" % (n_out, q))
+    rng = np.random.default_rng(2600 + q + tiles)
+    xb = (rng.random((70000 // n + 3, n), dtype=np.float32) * 2 - 1).astype(np.float32)
+    yb = run_1d(xb, ws[q], design, cuda_device, batch_stride=(n + 3) // 4 * 4)
+    for b in range(xb.shape[0]):
+        y_ref, s_ref = oracle.conv1d_f32(xb[b], ws[q])
+        assert_close_f32(yb[b], y_ref, s_ref, "batch %d" % b)
+    assert B.device_status() == 0
+
+
+@pytest.mark.parametrize("design", STRIDED_1D, ids=_ids)
+@pytest.mark.parametrize("q", [5, 8, 32])
+@pytest.mark.parametrize("tiles", [1, 2, 3, 4])
+def test_1d_stride2_output_count_a_whole_number_of_tiles(cuda_device, design, q, tiles):
+    n_out = 608 * tiles
+    for n in (2 * (n_out - 1) + q, 2 * (n_out - 1) + q + 1):
+        x, ws = inputs.gen_1d_f32(n, [q], seed=2700 + q + tiles)
+        y_ref, s_ref = oracle.conv1d_f32_strided(x, ws[q], 2)
+        assert y_ref.size == n_out
+        y = B.conv1d(torch.from_numpy(x).to(cuda_device), ws[q], design, stride=2)
+        torch.cuda.synchronize()
+        assert_close_f32(y.cpu().numpy(), y_ref, s_ref, "n=%d q=%d" % (n, q))
+        xb = np.stack([x, x[::-1].copy(), -x])
+        yd = B.conv1d(torch.from_numpy(xb).to(cuda_device), ws[q], design, stride=2)
+        torch.cuda.synchronize()
+        for b in range(3):
+            y_ref, s_ref = oracle.conv1d_f32_strided(xb[b], ws[q], 2)
+            assert_close_f32(yd[b].cpu().numpy(), y_ref, s_ref, "batch %d" % b)
     assert B.device_status() == 0
 
 
@@ -310,30 +352,42 @@ def test_config5_reduced_and_exact_integers(cuda_device, design, k):
 
 
 @pytest.mark.parametrize("k", [3, 9, 15])
-def test_config5_full_size_sampled(cuda_device, k):
-    """16 x 4096 x 4096 in the bench's launch configuration; sampled outputs against the oracle."""
+def test_config5_full_size_every_output(cuda_device, k):
+    """16 x 4096 x 4096 in the bench's launch configuration: EVERY output of every image, for the three designs,
+    against the oracle (one oracle pass per image, the three designs compared with it in turn)."""
     x, ws = inputs.make_config(5, scale=dict(filters=[k]))
     w = ws[(k, k)]
     xd = torch.from_numpy(x).to(cuda_device)
-    rng = np.random.default_rng(5)
     oh = ow = 4096 - k + 1
-    rows = np.concatenate([rng.integers(0, oh, 4000), [0, 0, oh - 1, oh - 1]]).astype(np.int64)
-    cols = np.concatenate([rng.integers(0, ow, 4000), [0, ow - 1, 0, ow - 1]]).astype(np.int64)
-    yd = torch.empty((16, oh, ow), dtype=torch.float32, device=cuda_device)
+    outs = {}
     for design in DESIGNS:
-        yd.fill_(CANARY)
-        B.conv2d(xd, w, design, out=yd)
-        torch.cuda.synchronize()
-        ri, ci = torch.from_numpy(rows).to(cuda_device), torch.from_numpy(cols).to(cuda_device)
-        for b in range(16):
-            got = yd[b][ri, ci].cpu().numpy()
-            y_ref, s_ref = oracle.conv2d_f32_at(x[b], w, rows, cols)
-            assert_close_f32(got, y_ref, s_ref, "config 5 k=%d design %s image %d" % (k, _ids(design), b))
-        # every output was written (no canary left) and the whole of image 7 matches at k = 3
-        assert not bool((yd == CANARY).any())
-        if k == 3:
-            y_ref, s_ref = oracle.conv2d_f32(x[7], w)
-            assert_close_f32(yd[7].cpu().numpy(), y_ref, s_ref, "config 5 image 7 full")
+        # pitch rounded up to 4 elements, as bench.py allocates its outputs; the padding keeps its canary
+        yd = torch.full((16, oh, (ow + 3) // 4 * 4), CANARY, dtype=torch.float32, device=cuda_device)
+        B.conv2d(xd, w, design, out=yd[:, :, :ow])
+        outs[design] = yd
+    torch.cuda.synchronize()
+    del xd
+    for b in range(16):
+        y_ref, s_ref = oracle.conv2d_f32(x[b], w)
+        for design in DESIGNS:
+            got = outs[design][b].cpu().numpy()
+            assert (got[:, ow:] == CANARY).all(), "write into the pitch padding"
+            assert_close_f32(got[:, :ow], y_ref, s_ref, "config 5 k=%d design %s image %d" % (k, _ids(design), b))
+
+
+# The fp32 OS / IS kernels for small filters (P*Q <= 25) have a form with eight PEs per lane that only large
+# problems reach (256-column strips x images x 8-row groups >= 4736); these cases are sized for it, with a ragged
+# right edge and a ragged last band.
+@pytest.mark.parametrize("design", [B.OS, B.IS], ids=_ids)
+@pytest.mark.parametrize("pq", [(5, 5), (2, 11), (1, 15), (4, 6), (3, 8), (5, 4), (1, 1), (2, 2), (3, 3), (12, 2), (15, 1)],
+                         ids=lambda f: "%dx%d" % f)
+def test_2d_f32_small_filters_eight_pes_per_lane(cuda_device, design, pq):
+    p, q = pq
+    wd, h, batch = 1301, 803, 8
+    assert ((wd - q + 1 + 255) // 256) * batch * ((h - p + 1 + 7) // 8) >= 4736
+    x, ws = inputs.gen_2d_f32(wd, h, [pq], seed=1200 + 16 * p + q, batch=batch)
+    check_2d(x, ws[pq], design, cuda_device)
+    check_2d(x[:6, :, :1290], ws[pq], design, cuda_device, x_pitch=1292, y_pitch=1292, x_off=4, y_off=4)
 
 
 # ------------------------------------------------------------------------ non-finite inputs
@@ -585,7 +639,7 @@ def check_separable(x_np, u, v, device, x_pitch=None, y_pitch=None, x_off=0, y_o
     for b in range(batch):
         # the definition: Eq. 3 with the rank-one filter u v^T (fp32 product of the taps, as the oracle takes fp32 taps)
         y_ref, s_ref = oracle.conv2d_f32(x_np[b], w)
-        assert_close_f32(body[b, :, :ow], y_ref, 1.0001 * s_ref + 1e-30, "image %d" % b)
+        assert_close_f32(body[b, :, :ow], y_ref, s_ref, "image %d" % b)
 
 
 @pytest.mark.parametrize("pq", [(1, 1), (3, 3), (5, 5), (7, 7), (8, 8), (9, 9), (15, 15), (2, 11), (13, 4), (15, 1), (1, 15),
@@ -636,7 +690,7 @@ def test_separable_full_size_sampled(cuda_device):
     rows = np.concatenate([rng.integers(0, oh, 3000), [0, 0, oh - 1, oh - 1]])
     cols = np.concatenate([rng.integers(0, ow, 3000), [0, ow - 1, 0, ow - 1]])
     y_ref, s_ref = oracle.conv2d_f32_at(x[1], np.outer(u.astype(np.float64), v.astype(np.float64)).astype(np.float32), rows, cols)
-    assert_close_f32(y[1].cpu().numpy()[rows, cols], y_ref, 1.0001 * s_ref + 1e-30, "sampled")
+    assert_close_f32(y[1].cpu().numpy()[rows, cols], y_ref, s_ref, "sampled")
 
 
 # ------------------------------------------------------------------------ generic space-time executor
@@ -723,6 +777,29 @@ def test_host_multi_entry_point(cuda_device):
         for (w, d, yh), q in zip(jobs, qs):
             y_ref, s_ref = oracle.conv1d_f32(x, w)
             assert_close_f32(yh.numpy(), y_ref, s_ref, "n=%d q=%d %s" % (n, q, B.DESIGN_NAMES[d]))
+    assert B.device_status() == 0
+
+
+# ------------------------------------------------------------------------ bounded device-side waits
+
+
+def test_a_bounded_wait_that_runs_out_is_reported_once(cuda_device):
+    """The pipelined kernels poll for their asynchronous copies a bounded number of times; a block whose limit runs
+    out raises a flag and returns.  The self-test block waits for bytes that are never sent (it issues no copy), so
+    its limit must run out: the launch completes, the status call reports the time-out once, then the device is
+    clean again and ordinary work runs."""
+    assert B.device_status() == 0
+    B.selftest_wait_timeout()
+    torch.cuda.synchronize()                       # the block returned by itself
+    assert B.device_status() == 4
+    assert B.device_status() == 0
+    side = torch.cuda.Stream()                     # a stream the legacy default stream does not wait for
+    B.selftest_wait_timeout(stream=side)
+    assert B.device_status() == 4                  # the status call synchronises the whole device itself
+    assert B.device_status() == 0
+    x, ws = inputs.make_config(1)
+    y_ref, s_ref = oracle.conv1d_f32(x, ws[8])
+    assert_close_f32(run_1d(x, ws[8], B.OS, cuda_device), y_ref, s_ref, "after the self-test")
     assert B.device_status() == 0
 
 

@@ -5,7 +5,8 @@ owns all device memory, a real-time loop with an allocation ban), so they cannot
 the device workspace it needs.  The static variant stages through a fixed array inside the library.
 This test calls it through the C ABI twice in a row -- the second call on a shorter, different signal
 with another design, so stale contents of the shared array would show -- and compares each result with
-what sysconv1d_host returns for the same inputs.
+what sysconv1d_host returns for the same inputs (same kernel, so the two must agree bit for bit) and
+with the CPU oracle (within the tolerance of the parity tests).
 
 Collected last on purpose: a failure here must not hide the other tests behind `-x`.
 """
@@ -13,6 +14,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2010_15884_b200 import binding as B
 from paper_2010_15884_b200 import inputs
 
@@ -34,10 +36,15 @@ def _both_ways(x, w, design, device):
     torch.cuda.synchronize()
     a, b = y_static.numpy().astype(np.float64), y_plain.numpy().astype(np.float64)
     assert np.isfinite(a).all() and np.isfinite(b).all()
-    # tolerance of the parity tests: 1e-5 * sum |w||x| per output
-    scale = np.stack([np.correlate(np.abs(row).astype(np.float64), np.abs(w).astype(np.float64), "valid")
-                      for row in x.reshape(-1, n)]).reshape(shape)
+    # against the existing entry point: within the tolerance of the parity tests, 1e-5 * sum |w||x| per output
+    # (both run the same kernel on the same data, so in fact every bit must agree)
+    ref = [oracle.conv1d_f32(row, w) for row in x.reshape(-1, n)]
+    y_ref = np.stack([r[0] for r in ref]).reshape(shape)
+    scale = np.stack([r[1] for r in ref]).reshape(shape)
     assert np.all(np.abs(a - b) <= TOL * scale)
+    assert np.array_equal(y_static.numpy(), y_plain.numpy())
+    # against the definition (Eq. 2), computed by the CPU oracle
+    assert np.all(np.abs(a - y_ref) <= TOL * scale)
 
 
 def test_static_variant_matches_workspace_variant_twice_in_a_row(cuda_device):
