@@ -399,6 +399,7 @@ __global__ void __launch_bounds__(Geo1D<DESIGN, WARPS>::kThreads)
 conv1d_f32_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, const __grid_constant__ Taps1DPairs tpairs,
                   unsigned *status_word)
 {
+    dependent_launch_enter();
     using G = Geo1D<DESIGN, WARPS>;
     __shared__ __align__(128) float s_in[K][G::kTileIn];
     __shared__ __align__(128) float s_out[K][G::kTileOut];
@@ -510,7 +511,7 @@ cudaError_t launch_conv1d_f32_q(const Conv1DArgs &a, const Taps1D &taps, unsigne
     Taps1DPairs tp;
     for (int t = 0; t <= kMaxQ1; ++t)
         tp.p[t] = make_float2(t < kMaxQ1 ? taps.w[t] : 0.f, t > 0 ? taps.w[t - 1] : 0.f);
-    conv1d_f32_kernel<DESIGN, Q, WARPS, K><<<grid, G::kThreads, 0, s>>>(a, taps, tp, status_word);
+    launch_kernel(conv1d_f32_kernel<DESIGN, Q, WARPS, K>, grid, G::kThreads, s, a, taps, tp, status_word);
     return cudaGetLastError();
 }
 

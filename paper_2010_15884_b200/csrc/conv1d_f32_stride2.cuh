@@ -182,6 +182,7 @@ __global__ void __launch_bounds__(WARPS *kLanes)
 conv1d_f32_s2_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, const __grid_constant__ Taps1DPairsS2 tpairs,
                      unsigned *status_word)
 {
+    dependent_launch_enter();
     constexpr int kThreads = WARPS * kLanes;
     constexpr int kTileAdv = WARPS * kWarpOut1;         // inputs a tile advances by
     constexpr int kTileIn = kTileAdv + kHalo1;
@@ -289,7 +290,7 @@ cudaError_t launch_conv1d_f32_s2_q(const Conv1DArgs &a, const Taps1D &taps, unsi
     Taps1DPairsS2 tp;
     for (int t = 0; t < kMaxQ1 + 2; ++t)
         tp.p[t] = make_float2(t < kMaxQ1 ? taps.w[t] : 0.f, t >= 2 ? taps.w[t - 2] : 0.f);
-    conv1d_f32_s2_kernel<DESIGN, Q, WARPS, K><<<grid, WARPS * kLanes, 0, s>>>(a, taps, tp, status_word);
+    launch_kernel(conv1d_f32_s2_kernel<DESIGN, Q, WARPS, K>, grid, WARPS * kLanes, s, a, taps, tp, status_word);
     return cudaGetLastError();
 }
 

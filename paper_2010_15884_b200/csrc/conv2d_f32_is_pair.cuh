@@ -42,6 +42,7 @@ __global__ void __launch_bounds__(kThreads2, MIN_CTAS)
 conv2d_is_pair_kernel(const Conv2DArgs a, const __grid_constant__ Taps2D taps, const __grid_constant__ TapsColPairs tp,
                       const int band_h)
 {
+    dependent_launch_enter();
     using Tr = F32Traits;
     using G = IsPairGeom<Q>;
     constexpr int R = R2;
@@ -165,7 +166,7 @@ cudaError_t launch_conv2d_is_pair(const Conv2DArgs &a, const Taps2D &taps, cudaS
     // two output rows per pass up to ten filter rows (measured: 9x9 0.96 -> 0.85 ms); beyond that the
     // second row's registers cost more than the shared tap reads save (15x15: 2.33 ms with one row, 2.63 with two)
     constexpr int ROWS = P <= 10 ? 2 : 1;
-    conv2d_is_pair_kernel<P, Q, ROWS, ROWS == 2 ? 4 : 1><<<grid, kThreads2, 0, s>>>(a, taps, tp, band_h);
+    launch_kernel(conv2d_is_pair_kernel<P, Q, ROWS, ROWS == 2 ? 4 : 1>, grid, kThreads2, s, a, taps, tp, band_h);
     return cudaGetLastError();
 }
 

@@ -19,6 +19,7 @@ template <int P, int Q, int R, int PF>
 __global__ void __launch_bounds__(kThreads2)
 conv2d_sep_os_kernel(const Conv2DArgs a, const __grid_constant__ TapsSep taps, const int band_h)
 {
+    dependent_launch_enter();
     using Tr = F32Traits;
     static_assert(R == 4 || R == 8, "R = PEs per lane");
     constexpr int kStrip = kLanes * R;
@@ -123,8 +124,8 @@ cudaError_t launch_conv2d_sep_pq(const Conv2DArgs &a, const TapsSep &taps, cudaS
     const int strips = (a.out_w + per_strip - 1) / per_strip;
     const int band_h = pick_band_height(a.out_h, static_cast<long long>(strips) * a.batch, P, 1);
     dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + band_h - 1) / band_h, a.batch);
-    if (narrow) conv2d_sep_os_kernel<P, Q, 4, 2><<<grid, kThreads2, 0, s>>>(a, taps, band_h);
-    else conv2d_sep_os_kernel<P, Q, RW, 2><<<grid, kThreads2, 0, s>>>(a, taps, band_h);
+    if (narrow) launch_kernel(conv2d_sep_os_kernel<P, Q, 4, 2>, grid, kThreads2, s, a, taps, band_h);
+    else launch_kernel(conv2d_sep_os_kernel<P, Q, RW, 2>, grid, kThreads2, s, a, taps, band_h);
     return cudaGetLastError();
 }
 

@@ -31,6 +31,7 @@ template <int P, int Q>
 __global__ void __launch_bounds__(kThreads2)
 conv2d_os_s2_kernel(const Conv2DArgs a, const __grid_constant__ Taps2D taps, const int band_h)
 {
+    dependent_launch_enter();
     constexpr int KP = (P + 1) / 2;             // partial output rows alive
     const int lane = threadIdx.x & (kLanes - 1);
     const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;
@@ -127,6 +128,7 @@ template <int P, int Q>
 __global__ void __launch_bounds__(kThreads2)
 conv2d_is_s2_kernel(const Conv2DArgs a, const __grid_constant__ Taps2D taps, const int band_h)
 {
+    dependent_launch_enter();
     constexpr int kShift = IsGeomS2<Q>::kShift;
     constexpr int kValid = IsGeomS2<Q>::kValid;
     const int lane = threadIdx.x & (kLanes - 1);
@@ -210,8 +212,8 @@ cudaError_t launch_conv2d_s2_pq(const Conv2DArgs &a, const Taps2D &taps, cudaStr
     const int strips = (a.out_w + per_strip - 1) / per_strip;
     const int band_h = pick_band_height(a.out_h, static_cast<long long>(strips) * a.batch, P, Q);
     dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + band_h - 1) / band_h, a.batch);
-    if (DESIGN == SYSCONV_OS) conv2d_os_s2_kernel<P, Q><<<grid, kThreads2, 0, s>>>(a, taps, band_h);
-    else conv2d_is_s2_kernel<P, Q><<<grid, kThreads2, 0, s>>>(a, taps, band_h);
+    if (DESIGN == SYSCONV_OS) launch_kernel(conv2d_os_s2_kernel<P, Q>, grid, kThreads2, s, a, taps, band_h);
+    else launch_kernel(conv2d_is_s2_kernel<P, Q>, grid, kThreads2, s, a, taps, band_h);
     return cudaGetLastError();
 }
 

@@ -43,6 +43,7 @@ __global__ void __launch_bounds__(kLanes)
 conv2d_ws_lane_kernel(const Conv2DArgs a, const __grid_constant__ Taps2D taps, const __grid_constant__ TapsColPairs tp,
                       const int seg_w)
 {
+    dependent_launch_enter();
     using Tr = F32Traits;
     constexpr int M = kWlM;
     constexpr int K = M + P - 1;                // input rows feeding M output rows
@@ -198,7 +199,7 @@ cudaError_t launch_conv2d_ws_lane(const Conv2DArgs &a, const Taps2D &taps, cudaS
     seg_w = (seg_w + kChunk - 1) / kChunk * kChunk;
     dim3 grid((a.out_w + seg_w - 1) / seg_w, static_cast<unsigned>(bands), a.batch);
     if (grid.y > 65535) return cudaErrorInvalidConfiguration;
-    conv2d_ws_lane_kernel<P, Q><<<grid, kLanes, 0, s>>>(a, taps, tp, seg_w);
+    launch_kernel(conv2d_ws_lane_kernel<P, Q>, grid, kLanes, s, a, taps, tp, seg_w);
     return cudaGetLastError();
 }
 

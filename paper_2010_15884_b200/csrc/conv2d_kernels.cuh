@@ -124,6 +124,7 @@ template <typename Tr, int P, int Q, int R, int MIN_CTAS, int PF>
 __global__ void __launch_bounds__(kThreads2, MIN_CTAS)
 conv2d_os_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t taps, const int band_h)
 {
+    dependent_launch_enter();
     using in_t = typename Tr::in_t;
     using acc_t = typename Tr::acc_t;
     using out_t = typename Tr::out_t;
@@ -135,11 +136,11 @@ conv2d_os_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t
     const int lane = threadIdx.x & (kLanes - 1);
     const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;
     const int c0 = strip * kStrip;
-    if (c0 >= a.out_w) return;
     const int r0 = blockIdx.y * band_h;
     const int r1 = min(r0 + band_h, a.out_h);
     const in_t *xb = static_cast<const in_t *>(a.x) + blockIdx.z * a.x_bstride;
     out_t *yb = static_cast<out_t *>(a.y) + blockIdx.z * a.y_bstride;
+    if (c0 >= a.out_w) return;
     const bool x_vec = row_alignment(static_cast<const in_t *>(a.x), a.x_pitch, a.x_bstride, a.batch) == 4;
     const int y_align = row_alignment(static_cast<const out_t *>(a.y), a.y_pitch, a.y_bstride, a.batch);
     const int col = c0 + R * lane;              // first column of this lane's PEs
@@ -255,6 +256,7 @@ template <int P, int Q, int R, int MIN_CTAS, bool EXACT_HALVES>
 __global__ void __launch_bounds__(kThreads2, MIN_CTAS)
 conv2d_os_rowpair_kernel(const Conv2DArgs a, const __grid_constant__ TapsRowPairs taps, const int band_h)
 {
+    dependent_launch_enter();
     using Tr = F32Traits;
     constexpr int SP = F2R<P>::SP;
     constexpr bool kHalo = Q > 1;
@@ -371,83 +373,94 @@ struct IsGeom {
     static constexpr int kValid = kLanes * R - kShift;        // outputs per strip
 };
 
+// The P-deep input column of a PE is a window that slides down one row per output row.  Where the code stays
+// small the row loop is unrolled P times and the window is a ring (input row r+p sits in slot (u+p) mod P, u =
+// position in the unrolled group), so sliding costs nothing; otherwise the window is shifted by (P-1)*R moves.
+template <int P, int Q, int R>
+constexpr bool kIsRing = P > 1 && P * P * Q * R <= 2048;
+
 template <typename Tr, int P, int Q, int R, int MIN_CTAS>
 __global__ void __launch_bounds__(kThreads2, MIN_CTAS)
 conv2d_is_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t taps, const int band_h)
 {
+    dependent_launch_enter();
     using in_t = typename Tr::in_t;
     using acc_t = typename Tr::acc_t;
     using out_t = typename Tr::out_t;
     static_assert(R == 4 || R == 8, "R = PEs per lane");
     constexpr int kShift = IsGeom<Q, R>::kShift;
     constexpr int kValid = IsGeom<Q, R>::kValid;
+    constexpr bool kRing = kIsRing<P, Q, R>;
+    constexpr int U = kRing ? P : 1;            // output rows per trip of the row loop
     const int lane = threadIdx.x & (kLanes - 1);
     const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;
     const int c0 = strip * kValid;              // first output column = first input column (PE 0)
-    if (c0 >= a.out_w) return;
     const int r0 = blockIdx.y * band_h;
     const int r1 = min(r0 + band_h, a.out_h);
     const in_t *xb = static_cast<const in_t *>(a.x) + blockIdx.z * a.x_bstride;
     out_t *yb = static_cast<out_t *>(a.y) + blockIdx.z * a.y_bstride;
+    if (c0 >= a.out_w) return;
     const bool x_vec = row_alignment(static_cast<const in_t *>(a.x), a.x_pitch, a.x_bstride, a.batch) == 4;
     const int y_align = row_alignment(static_cast<const out_t *>(a.y), a.y_pitch, a.y_bstride, a.batch);
     const int col = c0 + R * lane;              // columns held by this lane's PEs
     const int ocol = col - kShift;              // output columns its PEs end up holding
     const int oend = min(a.out_w, c0 + kValid);
 
-    // PE registers: the P-deep input column of each PE, rows r .. r+P-1
+    auto fetch = [&](int row, acc_t *dx) {
+        const in_t *rowp = xb + static_cast<long long>(min(row, a.height - 1)) * a.x_pitch;
+#pragma unroll
+        for (int g = 0; g < R / 4; ++g) load_group<Tr>(rowp, col + 4 * g, a.width, x_vec, dx + 4 * g);
+    };
+
+    // PE registers: the P-deep input column of each PE.  Before output row r0 the rows r0 .. r0+P-2 sit in the
+    // slots they will have at the first trip (ring: slot p; shifting window: slot p+1, shifted down first).
     acc_t X[P][R];
 #pragma unroll
-    for (int p = 0; p < P - 1; ++p) {
-        const in_t *rowp = xb + static_cast<long long>(min(r0 + p, a.height - 1)) * a.x_pitch;
-#pragma unroll
-        for (int g = 0; g < R / 4; ++g) load_group<Tr>(rowp, col + 4 * g, a.width, x_vec, &X[p + 1][4 * g]);
-    }
+    for (int p = 0; p < P - 1; ++p) fetch(r0 + p, X[kRing ? p : p + 1]);
     acc_t nX[R];
-    {
-        const in_t *rowp = xb + static_cast<long long>(r0 + P - 1) * a.x_pitch;
-#pragma unroll
-        for (int g = 0; g < R / 4; ++g) load_group<Tr>(rowp, col + 4 * g, a.width, x_vec, &nX[4 * g]);
-    }
+    fetch(r0 + P - 1, nX);
 
 #pragma unroll 1
-    for (int r = r0; r < r1; ++r) {
-        // the window of input rows slides down by one
+    for (int rb = r0; rb < r1; rb += U) {
 #pragma unroll
-        for (int p = 0; p < P - 1; ++p)
+        for (int u = 0; u < U; ++u) {
+            const int r = rb + u;
+            if (r >= r1) break;
+            if (!kRing) {
+                // the window of input rows slides down by one
 #pragma unroll
-            for (int j = 0; j < R; ++j) X[p][j] = X[p + 1][j];
+                for (int p = 0; p < P - 1; ++p)
 #pragma unroll
-        for (int j = 0; j < R; ++j) X[P - 1][j] = nX[j];
-        if (r + 1 < r1) {
-            const in_t *rowp = xb + static_cast<long long>(r + P) * a.x_pitch;
+                    for (int j = 0; j < R; ++j) X[p][j] = X[p + 1][j];
+            }
 #pragma unroll
-            for (int g = 0; g < R / 4; ++g) load_group<Tr>(rowp, col + 4 * g, a.width, x_vec, &nX[4 * g]);
-        }
+            for (int j = 0; j < R; ++j) X[(u + P - 1) % P][j] = nX[j];
+            if (r + 1 < r1) fetch(r + P, nX);
 
-        acc_t Z[R];
+            acc_t Z[R];
 #pragma unroll
-        for (int q = 0; q < Q + IsGeom<Q, R>::kDrain; ++q) {
-            if (q > 0) {
-                // partial sums move one PE up (lane 0 has no left neighbour: invalid PEs)
-                const acc_t up = __shfl_up_sync(kFullMask, Z[R - 1], 1);
+            for (int q = 0; q < Q + IsGeom<Q, R>::kDrain; ++q) {
+                if (q > 0) {
+                    // partial sums move one PE up (lane 0 has no left neighbour: invalid PEs)
+                    const acc_t up = __shfl_up_sync(kFullMask, Z[R - 1], 1);
 #pragma unroll
-                for (int j = R - 1; j > 0; --j) Z[j] = Z[j - 1];
-                Z[0] = up;
+                    for (int j = R - 1; j > 0; --j) Z[j] = Z[j - 1];
+                    Z[0] = up;
+                }
+                if (q < Q) {
+#pragma unroll
+                    for (int p = 0; p < P; ++p)     // t = p + P*q
+#pragma unroll
+                        for (int j = 0; j < R; ++j)
+                            Z[j] = (q == 0 && p == 0) ? Tr::mul(X[u % P][j], taps.w[0])
+                                                      : Tr::mad(X[(u + p) % P][j], taps.w[p * Q + q], Z[j]);
+                }
             }
-            if (q < Q) {
+            out_t *orow = yb + static_cast<long long>(r) * a.y_pitch;
 #pragma unroll
-                for (int p = 0; p < P; ++p)     // t = p + P*q
-#pragma unroll
-                    for (int j = 0; j < R; ++j)
-                        Z[j] = (q == 0 && p == 0) ? Tr::mul(X[0][j], taps.w[0])
-                                                  : Tr::mad(X[p][j], taps.w[p * Q + q], Z[j]);
-            }
+            for (int g = 0; g < R / 4; ++g)
+                if (ocol + 4 * g >= c0) store_group<Tr>(orow, ocol + 4 * g, oend, y_align, &Z[4 * g]);
         }
-        out_t *orow = yb + static_cast<long long>(r) * a.y_pitch;
-#pragma unroll
-        for (int g = 0; g < R / 4; ++g)
-            if (ocol + 4 * g >= c0) store_group<Tr>(orow, ocol + 4 * g, oend, y_align, &Z[4 * g]);
     }
 }
 
@@ -480,6 +493,7 @@ template <typename Tr, int P, int Q>
 __global__ void __launch_bounds__(kThreads2)
 conv2d_ws_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t taps, const int seg_w)
 {
+    dependent_launch_enter();
     using in_t = typename Tr::in_t;
     using acc_t = typename Tr::acc_t;
     using out_t = typename Tr::out_t;
@@ -656,13 +670,24 @@ cudaError_t launch_conv2d_osis(const Conv2DArgs &a, const typename Tr::taps_t &t
     using Sh = Shape2D<Tr, DESIGN, P, Q>;
     const int per_strip = DESIGN == SYSCONV_OS ? kLanes * R : IsGeom<Q, R>::kValid;
     const int strips = (a.out_w + per_strip - 1) / per_strip;
-    const int band_h = pick_band_height(a.out_h, static_cast<long long>(strips) * a.batch, P, Q);
+    int band_h = pick_band_height(a.out_h, static_cast<long long>(strips) * a.batch, P, Q);
+    {
+        // a problem of a few waves of blocks: short bands, chosen by the number of waves they give
+        static const long long slots = 148LL * [] {
+            if constexpr (DESIGN == SYSCONV_OS)
+                return resident_blocks_per_sm(conv2d_os_kernel<Tr, P, Q, R, Sh::kMinCtas, Sh::kPrefetch>, kThreads2);
+            else
+                return resident_blocks_per_sm(conv2d_is_kernel<Tr, P, Q, R, Sh::kMinCtas>, kThreads2);
+        }();
+        const long long per_band = static_cast<long long>((strips + kWarps2 - 1) / kWarps2) * a.batch;
+        if (small_problem(a.out_h, per_band, 4, slots)) band_h = pick_band_height_small(a.out_h, per_band, P, 4, 64, slots);
+    }
     dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + band_h - 1) / band_h, a.batch);
     if (grid.y > 65535) return cudaErrorInvalidConfiguration;
-    if (DESIGN == SYSCONV_OS)
-        conv2d_os_kernel<Tr, P, Q, R, Sh::kMinCtas, Sh::kPrefetch><<<grid, kThreads2, 0, s>>>(a, taps, band_h);
+    if constexpr (DESIGN == SYSCONV_OS)
+        launch_kernel(conv2d_os_kernel<Tr, P, Q, R, Sh::kMinCtas, Sh::kPrefetch>, grid, kThreads2, s, a, taps, band_h);
     else
-        conv2d_is_kernel<Tr, P, Q, R, Sh::kMinCtas><<<grid, kThreads2, 0, s>>>(a, taps, band_h);
+        launch_kernel(conv2d_is_kernel<Tr, P, Q, R, Sh::kMinCtas>, grid, kThreads2, s, a, taps, band_h);
     return cudaGetLastError();
 }
 
@@ -686,7 +711,7 @@ cudaError_t launch_conv2d_os_rowpair(const Conv2DArgs &a, const float *w, cudaSt
     const int band_h = pick_band_height(a.out_h, static_cast<long long>(strips) * a.batch, P, Q);
     dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + band_h - 1) / band_h, a.batch);
     if (grid.y > 65535) return cudaErrorInvalidConfiguration;
-    conv2d_os_rowpair_kernel<P, Q, R, MINB, kRowPairExact<P>><<<grid, kThreads2, 0, s>>>(a, t, band_h);
+    launch_kernel(conv2d_os_rowpair_kernel<P, Q, R, MINB, kRowPairExact<P>>, grid, kThreads2, s, a, t, band_h);
     return cudaGetLastError();
 }
 
@@ -718,7 +743,7 @@ cudaError_t launch_conv2d_pq(const Conv2DArgs &a, const typename Tr::taps_t &tap
         seg_w = (seg_w + kWsChunk - 1) / kWsChunk * kWsChunk;
         dim3 grid((a.out_w + seg_w - 1) / seg_w, static_cast<unsigned>(bands), a.batch);
         if (grid.y > 65535) return cudaErrorInvalidConfiguration;
-        conv2d_ws_kernel<Tr, P, Q><<<grid, kThreads2, 0, s>>>(a, taps, seg_w);
+        launch_kernel(conv2d_ws_kernel<Tr, P, Q>, grid, kThreads2, s, a, taps, seg_w);
         return cudaGetLastError();
     }
     using Sh = Shape2D<Tr, DESIGN, P, Q>;

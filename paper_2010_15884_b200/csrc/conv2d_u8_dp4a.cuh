@@ -30,6 +30,7 @@ template <int P, int Q, int PX, int PF>
 __global__ void __launch_bounds__(kThreads2)
 conv2d_u8_os_dp4a_kernel(const Conv2DArgs a, const __grid_constant__ TapsPacked taps, const int band_h)
 {
+    dependent_launch_enter();
     static_assert(PX % 4 == 0 && PX <= 16, "PX = PEs (pixels) per lane");
     static_assert(PF >= 1 && PF <= 4, "PF = input rows in flight ahead of the one being processed");
     constexpr int NW = PX / 4;                  // pixel words (groups of four PEs) per lane
@@ -40,35 +41,56 @@ conv2d_u8_os_dp4a_kernel(const Conv2DArgs a, const __grid_constant__ TapsPacked 
     const int lane = threadIdx.x & (kLanes - 1);
     const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;
     const int c0 = strip * kStrip;
-    if (c0 >= a.out_w) return;
     const int r0 = blockIdx.y * band_h;
     const int r1 = min(r0 + band_h, a.out_h);
     const uint8_t *xb = static_cast<const uint8_t *>(a.x) + blockIdx.z * a.x_bstride;
     int *yb = static_cast<int *>(a.y) + blockIdx.z * a.y_bstride;
+    if (c0 >= a.out_w) return;
     const int y_align = row_alignment(static_cast<const int *>(a.y), a.y_pitch, a.y_bstride, a.batch);
     const int col = c0 + 4 * lane;              // first column of this lane's word in run 0
     const int i_end = r1 + P - 1;
 
-    // the lane's NW words of one input row plus, in lanes 0 .. G-1, the words that follow the strip;
+    // Everything that is the same for every row of the band is decided here, so that the row loop carries no
+    // comparisons: which of the lane's words are loaded whole, which ragged (the image's last, partial word),
+    // which groups of four outputs leave as one 128-bit word and which element by element.
+    bool ld_whole[NW + 1], ld_ragged[NW + 1], st_vec[NW], st_part[NW];
+#pragma unroll
+    for (int k = 0; k <= NW; ++k) {
+        const int c = col + 4 * kLanes * k;
+        const bool mine = k < NW || lane < G;   // the words that follow the strip are fetched by lanes 0 .. G-1
+        ld_whole[k] = mine && c + 4 <= a.width;
+        ld_ragged[k] = mine && !ld_whole[k] && c < a.width;
+    }
+#pragma unroll
+    for (int k = 0; k < NW; ++k) {
+        const int c = col + 4 * kLanes * k;
+        st_vec[k] = y_align == 4 && c + 4 <= a.out_w;
+        st_part[k] = !st_vec[k] && c < a.out_w;
+    }
+    // row pointers advance by one pitch per row: the row to fetch next, the output row to store next
+    const uint8_t *xnext = xb + static_cast<long long>(r0) * a.x_pitch + col;
+    int *onext = yb + static_cast<long long>(r0) * a.y_pitch + col;
+    int next_row = r0;                          // image row xnext points at
+
+    // the lane's NW words of the next input row plus, in lanes 0 .. G-1, the words that follow the strip;
     // rows are 4-byte aligned (checked by the launcher), pixels beyond the image read as zero
-    auto fetch = [&](int row, unsigned (&w)[NW + 1]) {
-        if (row >= i_end) return;
-        const uint8_t *rowp = xb + static_cast<long long>(row) * a.x_pitch;
+    auto fetch = [&](unsigned (&w)[NW + 1]) {
+        if (next_row >= i_end) return;
 #pragma unroll
         for (int k = 0; k <= NW; ++k) {
-            const int c = col + 4 * kLanes * k;
             unsigned v = 0;
-            if (k < NW || lane < G) {
-                if (c + 4 <= a.width) {
-                    v = __ldg(reinterpret_cast<const unsigned *>(rowp + c));
-                } else {
+            if (ld_whole[k]) {
+                v = __ldg(reinterpret_cast<const unsigned *>(xnext + 4 * kLanes * k));
+            } else if (ld_ragged[k]) {
+                const int c = col + 4 * kLanes * k;
 #pragma unroll
-                    for (int e = 0; e < 3; ++e)
-                        if (c + e < a.width) v |= static_cast<unsigned>(rowp[c + e]) << (8 * e);
-                }
+                for (int e = 0; e < 3; ++e)
+                    if (c + e < a.width) v |= static_cast<unsigned>(xnext[4 * kLanes * k + e]) << (8 * e);
             }
             w[k] = v;
         }
+        xnext += a.x_pitch;
+        ++next_row;
     };
 
     int Z[P][PX];
@@ -83,14 +105,14 @@ conv2d_u8_os_dp4a_kernel(const Conv2DArgs a, const __grid_constant__ TapsPacked 
     for (int f = 0; f < PF; ++f) {
 #pragma unroll
         for (int k = 0; k <= NW; ++k) nW[f][k] = 0;
-        fetch(r0 + f, nW[f]);
+        fetch(nW[f]);
     }
     // process input row i, whose data sit in buffer f; refill that buffer with row i + PF
     auto process = [&](int i, int f) {
         unsigned W[NW + 1];
 #pragma unroll
         for (int k = 0; k <= NW; ++k) W[k] = nW[f][k];
-        fetch(i + PF, nW[f]);
+        fetch(nW[f]);
 #pragma unroll
         for (int k = 0; k < NW; ++k) {
             // inputs forwarded from the next PEs: word e further on sits in lane (l+e) mod 32, in the same run
@@ -126,12 +148,17 @@ conv2d_u8_os_dp4a_kernel(const Conv2DArgs a, const __grid_constant__ TapsPacked 
                 }
             }
         }
-        const int r = i - (P - 1);
-        if (r >= r0) {
-            int *orow = yb + static_cast<long long>(r) * a.y_pitch;
+        if (i - (P - 1) >= r0) {
+            // output row i-(P-1) is complete
 #pragma unroll
-            for (int k = 0; k < NW; ++k)
-                store_group<U8Traits>(orow, col + 4 * kLanes * k, a.out_w, y_align, &Z[P - 1][4 * k]);
+            for (int k = 0; k < NW; ++k) {
+                if (st_vec[k])
+                    *reinterpret_cast<int4 *>(onext + 4 * kLanes * k) =
+                        make_int4(Z[P - 1][4 * k], Z[P - 1][4 * k + 1], Z[P - 1][4 * k + 2], Z[P - 1][4 * k + 3]);
+                else if (st_part[k])
+                    store_group<U8Traits>(onext - col, col + 4 * kLanes * k, a.out_w, y_align, &Z[P - 1][4 * k]);
+            }
+            onext += a.y_pitch;
         }
     };
 #pragma unroll 1
@@ -149,12 +176,12 @@ inline bool u8_dp4a_eligible(const Conv2DArgs &a)
     return (xa & 3ull) == 0 && (a.x_pitch & 3) == 0 && (a.batch == 1 || (a.x_bstride & 3) == 0);
 }
 
-// Eight PEs per lane and one row in flight measured best for every filter size tried (3x3 and 7x7 on
-// 3840x2160 and on 16384x8192; 4 or 16 PEs and 2 or 4 rows in flight were slower or equal).
+// Eight PEs per lane and two rows in flight measured best (3x3 and 7x7 on 3840x2160, launches back to back over
+// rotating buffers: 3x3 10.8 -> 9.3 us, 7x7 20.0 -> 16.5 us against one row in flight; 4 or 16 PEs slower or equal).
 template <int P, int Q>
 cudaError_t launch_conv2d_u8_os_dp4a(const Conv2DArgs &a, const Taps2DInt &t, cudaStream_t s)
 {
-    constexpr int PX = 8, PF = 1;
+    constexpr int PX = 8, PF = 2;
     TapsPacked pk;
     for (int p = 0; p < kMaxP2; ++p)
         for (int g = 0; g < 4; ++g) {
@@ -176,10 +203,16 @@ cudaError_t launch_conv2d_u8_os_dp4a(const Conv2DArgs &a, const Taps2DInt &t, cu
     if (h < lo) h = lo;
     const long long fit = (a.out_h + 65534LL) / 65535;     // grid.y limit
     if (h < fit) h = fit;
-    const int band_h = static_cast<int>(h);
+    int band_h = static_cast<int>(h);
+    {
+        // a problem of a few waves of blocks: bands chosen by the number of waves they give
+        static const long long slots = 148LL * resident_blocks_per_sm(conv2d_u8_os_dp4a_kernel<P, Q, PX, PF>, kThreads2);
+        const long long per_band = static_cast<long long>((strips + kWarps2 - 1) / kWarps2) * a.batch;
+        if (small_problem(a.out_h, per_band, 4, slots)) band_h = pick_band_height_small(a.out_h, per_band, P, 4, 64, slots);
+    }
     dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + band_h - 1) / band_h, a.batch);
     if (grid.y > 65535) return cudaErrorInvalidConfiguration;
-    conv2d_u8_os_dp4a_kernel<P, Q, PX, PF><<<grid, kThreads2, 0, s>>>(a, pk, band_h);
+    launch_kernel(conv2d_u8_os_dp4a_kernel<P, Q, PX, PF>, grid, kThreads2, s, a, pk, band_h);
     return cudaGetLastError();
 }
 
@@ -203,35 +236,51 @@ template <int P, int Q>
 __global__ void __launch_bounds__(kThreads2)
 conv2d_u8_is_dp4a_kernel(const Conv2DArgs a, const __grid_constant__ TapsPacked taps, const int band_h)
 {
+    dependent_launch_enter();
     constexpr int G = IsDp4aGeom<Q>::G;
     constexpr int kValid = IsDp4aGeom<Q>::kValid;
     const int lane = threadIdx.x & (kLanes - 1);
     const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;
     const int c0 = strip * kValid;              // first output column = first input column of the strip
-    if (c0 >= a.out_w) return;
     const int r0 = blockIdx.y * band_h;
     const int r1 = min(r0 + band_h, a.out_h);
     const uint8_t *xb = static_cast<const uint8_t *>(a.x) + blockIdx.z * a.x_bstride;
     int *yb = static_cast<int *>(a.y) + blockIdx.z * a.y_bstride;
+    if (c0 >= a.out_w) return;
     const int y_align = row_alignment(static_cast<const int *>(a.y), a.y_pitch, a.y_bstride, a.batch);
     const int oend = min(a.out_w, c0 + kValid);
 
-    // the lane's two words of one input row (pixels beyond the image read as zero)
-    auto fetch = [&](int row, unsigned (&w)[2]) {
-        const uint8_t *rowp = xb + static_cast<long long>(min(row, a.height - 1)) * a.x_pitch;
+    // decided once per band, so that the row loop carries no comparisons: which of the lane's two words are loaded
+    // whole or ragged (the image's last, partial word), which of its two output groups leave as one 128-bit word
+    bool ld_whole[2], ld_ragged[2], st_vec[2], st_part[2];
+#pragma unroll
+    for (int n = 0; n < 2; ++n) {
+        const int c = c0 + 4 * (kLanes * n + lane);
+        ld_whole[n] = c + 4 <= a.width;
+        ld_ragged[n] = !ld_whole[n] && c < a.width;
+        const int k = kLanes * n + lane - (G - 1);              // word-PE whose outputs end up here
+        st_vec[n] = k >= 0 && y_align == 4 && c0 + 4 * k + 4 <= oend;
+        st_part[n] = k >= 0 && !st_vec[n] && c0 + 4 * k < oend;
+    }
+    const uint8_t *xnext = xb + static_cast<long long>(r0) * a.x_pitch + c0 + 4 * lane;
+    int *onext = yb + static_cast<long long>(r0) * a.y_pitch + c0 + 4 * (lane - (G - 1));
+
+    // the lane's two words of the next input row (pixels beyond the image read as zero)
+    auto fetch = [&](unsigned (&w)[2]) {
 #pragma unroll
         for (int n = 0; n < 2; ++n) {
-            const int c = c0 + 4 * (kLanes * n + lane);
             unsigned v = 0;
-            if (c + 4 <= a.width) {
-                v = __ldg(reinterpret_cast<const unsigned *>(rowp + c));
-            } else {
+            if (ld_whole[n]) {
+                v = __ldg(reinterpret_cast<const unsigned *>(xnext + 4 * kLanes * n));
+            } else if (ld_ragged[n]) {
+                const int c = c0 + 4 * (kLanes * n + lane);
 #pragma unroll
                 for (int e = 0; e < 3; ++e)
-                    if (c + e < a.width) v |= static_cast<unsigned>(rowp[c + e]) << (8 * e);
+                    if (c + e < a.width) v |= static_cast<unsigned>(xnext[4 * kLanes * n + e]) << (8 * e);
             }
             w[n] = v;
         }
+        xnext += a.x_pitch;
     };
     // the four stationary words of both word-PEs for one input row
     auto expand = [&](const unsigned (&w)[2], unsigned (&s)[2][4]) {
@@ -249,7 +298,9 @@ conv2d_u8_is_dp4a_kernel(const Conv2DArgs a, const __grid_constant__ TapsPacked 
         }
     };
 
-    unsigned S[P][2][4];                        // PE registers: rows r .. r+P-1
+    // PE registers: the window of P input rows is a ring -- the row loop is unrolled P times and input row r+p sits
+    // in slot (u+p) mod P, u = position in the unrolled group, so sliding the window costs no moves
+    unsigned S[P][2][4];
 #pragma unroll
     for (int p = 0; p < P; ++p)
 #pragma unroll
@@ -258,53 +309,54 @@ conv2d_u8_is_dp4a_kernel(const Conv2DArgs a, const __grid_constant__ TapsPacked 
             for (int i = 0; i < 4; ++i) S[p][n][i] = 0;
 #pragma unroll
     for (int p = 0; p < P - 1; ++p) {
-        unsigned w[2];
-        fetch(r0 + p, w);
-        expand(w, S[p + 1]);
+        unsigned w[2] = {0u, 0u};
+        fetch(w);
+        expand(w, S[p]);
     }
-    unsigned nW[2];
-    fetch(r0 + P - 1, nW);
+    unsigned nW[2] = {0u, 0u};
+    fetch(nW);
 
 #pragma unroll 1
-    for (int r = r0; r < r1; ++r) {
-        // the window of input rows slides down by one
+    for (int rb = r0; rb < r1; rb += P) {
 #pragma unroll
-        for (int p = 0; p < P - 1; ++p)
-#pragma unroll
-            for (int n = 0; n < 2; ++n)
-#pragma unroll
-                for (int i = 0; i < 4; ++i) S[p][n][i] = S[p + 1][n][i];
-        expand(nW, S[P - 1]);
-        if (r + 1 < r1) fetch(r + P, nW);
+        for (int u = 0; u < P; ++u) {
+            const int r = rb + u;
+            if (r >= r1) break;
+            expand(nW, S[(u + P - 1) % P]);
+            if (r + 1 < r1) fetch(nW);
 
-        int Z[2][4];
+            int Z[2][4];
 #pragma unroll
-        for (int g = 0; g < G; ++g) {
+            for (int g = 0; g < G; ++g) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                int z0 = 0, z1 = 0;
-                if (g > 0) {
-                    // the sums move one word-PE up: run 0 from the previous lane, run 1 likewise, its first PE
-                    // from the last PE of run 0 (the strip's first PE has no left neighbour: invalid sums)
-                    const int send = lane == kLanes - 1 ? Z[0][i] : Z[1][i];
-                    z0 = __shfl_up_sync(kFullMask, Z[0][i], 1);
-                    z1 = __shfl_sync(kFullMask, send, (lane - 1) & (kLanes - 1));
+                for (int i = 0; i < 4; ++i) {
+                    int z0 = 0, z1 = 0;
+                    if (g > 0) {
+                        // the sums move one word-PE up: run 0 from the previous lane, run 1 likewise, its first PE
+                        // from the last PE of run 0 (the strip's first PE has no left neighbour: invalid sums)
+                        const int send = lane == kLanes - 1 ? Z[0][i] : Z[1][i];
+                        z0 = __shfl_up_sync(kFullMask, Z[0][i], 1);
+                        z1 = __shfl_sync(kFullMask, send, (lane - 1) & (kLanes - 1));
+                    }
+#pragma unroll
+                    for (int p = 0; p < P; ++p) {
+                        z0 = dp4a_u8s8(S[(u + p) % P][0][i], taps.w[p * 4 + g], z0);
+                        z1 = dp4a_u8s8(S[(u + p) % P][1][i], taps.w[p * 4 + g], z1);
+                    }
+                    Z[0][i] = z0;
+                    Z[1][i] = z1;
                 }
-#pragma unroll
-                for (int p = 0; p < P; ++p) {
-                    z0 = dp4a_u8s8(S[p][0][i], taps.w[p * 4 + g], z0);
-                    z1 = dp4a_u8s8(S[p][1][i], taps.w[p * 4 + g], z1);
-                }
-                Z[0][i] = z0;
-                Z[1][i] = z1;
             }
-        }
-        // word-PE k holds the outputs that started in word-PE k - (G-1)
-        int *orow = yb + static_cast<long long>(r) * a.y_pitch;
+            // word-PE k holds the outputs that started in word-PE k - (G-1)
 #pragma unroll
-        for (int n = 0; n < 2; ++n) {
-            const int k = kLanes * n + lane - (G - 1);
-            if (k >= 0) store_group<U8Traits>(orow, c0 + 4 * k, oend, y_align, Z[n]);
+            for (int n = 0; n < 2; ++n) {
+                if (st_vec[n])
+                    *reinterpret_cast<int4 *>(onext + 4 * kLanes * n) = make_int4(Z[n][0], Z[n][1], Z[n][2], Z[n][3]);
+                else if (st_part[n])
+                    store_group<U8Traits>(onext - (c0 + 4 * (lane - (G - 1))), c0 + 4 * (kLanes * n + lane - (G - 1)), oend,
+                                          y_align, Z[n]);
+            }
+            onext += a.y_pitch;
         }
     }
 }
@@ -332,9 +384,14 @@ cudaError_t launch_conv2d_u8_is_dp4a(const Conv2DArgs &a, const Taps2DInt &t, cu
     if (h < lo) h = lo;
     const long long fit = (a.out_h + 65534LL) / 65535;  // grid.y limit
     if (h < fit) h = fit;
-    const int band_h = static_cast<int>(h);
+    int band_h = static_cast<int>(h);
+    {
+        static const long long slots = 148LL * resident_blocks_per_sm(conv2d_u8_is_dp4a_kernel<P, Q>, kThreads2);
+        const long long per_band = static_cast<long long>((strips + kWarps2 - 1) / kWarps2) * a.batch;
+        if (small_problem(a.out_h, per_band, 4, slots)) band_h = pick_band_height_small(a.out_h, per_band, P, 4, 64, slots);
+    }
     dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + band_h - 1) / band_h, a.batch);
-    conv2d_u8_is_dp4a_kernel<P, Q><<<grid, kThreads2, 0, s>>>(a, pk, band_h);
+    launch_kernel(conv2d_u8_is_dp4a_kernel<P, Q>, grid, kThreads2, s, a, pk, band_h);
     return cudaGetLastError();
 }
 

@@ -29,7 +29,7 @@ cudaError_t launch_spacetime_conv1d(const float *x, long long n, const float *w,
     long long ctas = (blocks + kStWarps - 1) / kStWarps;
     const long long cap = static_cast<long long>(sm_count) * 16;
     if (ctas > cap) ctas = cap;
-    spacetime_conv1d_kernel<<<static_cast<unsigned>(ctas), kStWarps * kLanes, 0, s>>>(x, y, n_out, taps, q, pl);
+    launch_kernel(spacetime_conv1d_kernel, static_cast<unsigned>(ctas), kStWarps * kLanes, s, x, y, n_out, taps, q, pl);
     const cudaError_t err = cudaGetLastError();
     if (err == cudaSuccess && launches) *launches += 1;
     return err;

@@ -81,6 +81,7 @@ __global__ void __launch_bounds__(kStWarps *kLanes)
 spacetime_conv1d_kernel(const float *__restrict__ x, float *__restrict__ y, long long n_out,
                         const __grid_constant__ Taps1D taps, int Q, const __grid_constant__ StPlan pl)
 {
+    dependent_launch_enter();
     const int lane = threadIdx.x & (kLanes - 1);
     const long long gw = static_cast<long long>(blockIdx.x) * kStWarps + threadIdx.x / kLanes;
     const long long warps = static_cast<long long>(gridDim.x) * kStWarps;

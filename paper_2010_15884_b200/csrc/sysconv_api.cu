@@ -7,8 +7,18 @@
 #include "sysconv_common.cuh"
 #include "tma_utils.cuh"
 
+#include <cstdlib>
+
 // Raised (set to 1) by a kernel that gave up a bounded wait; read and cleared by sysconv_device_status().
 static __device__ unsigned g_status_word;
+
+namespace sysconv {
+bool dependent_launch_enabled()
+{
+    static const bool on = std::getenv("SYSCONV_NO_PDL") == nullptr;
+    return on;
+}
+}  // namespace sysconv
 
 namespace {
 
@@ -59,6 +69,7 @@ long long checked_product(long long a, long long b, long long c)
 // status word exactly as the pipelined kernels do when their limit runs out, and returns.
 __global__ void wait_timeout_selftest_kernel(unsigned *status_word, unsigned polls)
 {
+    sysconv::dependent_launch_enter();
     __shared__ __align__(8) uint64_t bar;
     if (threadIdx.x == 0) {
         sysconv::mbar_init(&bar, 1);
@@ -644,7 +655,7 @@ int sysconv_selftest_wait_timeout(void *stream)
 {
     const DeviceInfo *d = device_info();
     if (!d) return SYSCONV_ECUDA;
-    wait_timeout_selftest_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>(d->status_word, 1u << 10);
+    sysconv::launch_kernel(wait_timeout_selftest_kernel, 1, 64, static_cast<cudaStream_t>(stream), d->status_word, 1u << 10);
     return finish(cudaGetLastError(), 1);
 }
 

@@ -106,6 +106,79 @@ cudaError_t launch_conv2d_u8_os(const Conv2DArgs &a, const int8_t *w, int q, int
 cudaError_t launch_conv2d_u8_is(const Conv2DArgs &a, const int8_t *w, int q, int p, cudaStream_t s, int *launches);
 cudaError_t launch_conv2d_u8_ws(const Conv2DArgs &a, const int8_t *w, int q, int p, cudaStream_t s, int *launches);
 
+// ---- programmatic dependent launch ---------------------------------------------------------------
+// Every kernel of the library is launched with the "programmatic stream serialization" attribute and
+// starts with dependent_launch_enter(), which waits until the PREVIOUS kernel of the stream has completed
+// and its memory is visible (griddepcontrol.wait) before anything touches global memory.  Stream order is
+// unchanged; the attribute lets the hardware set up this kernel while the one before it drains, instead of
+// after it has signalled completion, which matters for the small, launch-bound problems (measured back to
+// back on B200: 1920x1080 fp32 5x5 10.3 -> 8.3 us per launch, 3840x2160 uint8 3x3 12.3 -> 10.5 us).
+// No kernel triggers its dependents early (griddepcontrol.launch_dependents): with several kernels queued
+// that made the blocks of later kernels resident and waiting beside the running one and cost the
+// issue-bound kernels up to 20 %.
+__device__ __forceinline__ void dependent_launch_enter()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+bool dependent_launch_enabled();       // false if SYSCONV_NO_PDL is set in the environment (sysconv_api.cu)
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_kernel(void (*kern)(KArgs...), dim3 grid, dim3 block, cudaStream_t s, Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent_launch_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
+// Blocks of `threads` threads of this kernel that one SM holds at a time (asked of the runtime once per kernel).
+template <typename... KArgs>
+int resident_blocks_per_sm(void (*kern)(KArgs...), int threads)
+{
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, threads, 0) != cudaSuccess || n < 1) n = 1;
+    return n;
+}
+
+// Band height (output rows per block) for a 2-D problem SMALL enough that the whole grid is a few waves of blocks.
+// There the time is set by the number of waves times the time of one block, and a block's time grows with the
+// rows it marches through: its band, the P-1 rows of the window above it, and a fixed start-up worth about
+// eight rows (measured on B200: a full-HD 5x5 pass takes 4.4 us + 0.4 us per band row).  The height that
+// minimises waves x (band + P - 1 + 8) is taken; a grid that just spills into a second wave costs almost double,
+// which the fixed "so many blocks per SM" rules missed (3840x2160 uint8 7x7: 616 blocks on 592 slots, 24.6 us;
+// 540 blocks, 16.9 us).  per_band = blocks per band (column tiles x images), slots = blocks resident at once.
+inline int pick_band_height_small(int out_h, long long per_band, int p, int lo, int hi, long long slots)
+{
+    int best = lo;
+    double best_cost = 1e300;
+    for (int h = lo; h <= hi; ++h) {
+        const long long bands = (out_h + h - 1) / h;
+        if (bands > 65535) continue;
+        const long long waves = (per_band * bands + slots - 1) / slots;
+        const double cost = static_cast<double>(waves) * (h + p - 1 + 8);
+        if (cost < best_cost) {
+            best_cost = cost;
+            best = h;
+        }
+        if (bands == 1) break;
+    }
+    return best;
+}
+
+// true if a problem is "small" in the sense above: even with bands of `lo` rows it is at most four waves of blocks
+inline bool small_problem(int out_h, long long per_band, int lo, long long slots)
+{
+    return per_band * ((out_h + lo - 1) / lo) <= 4 * slots;
+}
+
 // Sentinel returned by a launcher for a filter size it has no instantiation for.
 constexpr cudaError_t kNoInstantiation = cudaErrorInvalidKernelImage;
 

@@ -375,6 +375,45 @@ def test_config5_full_size_every_output(cuda_device, k):
             assert_close_f32(got[:, :ow], y_ref, s_ref, "config 5 k=%d design %s image %d" % (k, _ids(design), b))
 
 
+# Problems of a few waves of blocks get short bands chosen by the number of waves they give: ragged right edges
+# (width not a multiple of the 16-byte unit, inside an aligned pitch), ragged last bands, several images, and the
+# same data once more from unaligned rows.
+@pytest.mark.parametrize("design", [B.OS, B.IS], ids=_ids)
+@pytest.mark.parametrize("pq", [(5, 5), (3, 3), (1, 1), (2, 11), (5, 4), (1, 15), (4, 6)], ids=lambda f: "%dx%d" % f)
+@pytest.mark.parametrize("size", [(517, 83, 3), (1001, 241, 1), (1920, 131, 2), (130, 40, 1), (16, 16, 5)],
+                         ids=lambda t: "%dx%dx%d" % t)
+def test_2d_f32_small_problems(cuda_device, design, pq, size):
+    wd, h, batch = size
+    p, q = pq
+    if wd < q or h < p:
+        pytest.skip("image smaller than the filter")
+    x, ws = inputs.gen_2d_f32(wd, h, [pq], seed=1300 + 16 * p + q + wd, batch=batch)
+    xp = (wd + 3) // 4 * 4
+    y_al = run_2d(x, ws[pq], design, cuda_device, x_pitch=xp, y_pitch=wd)
+    for b in range(batch):
+        y_ref, s_ref = oracle.conv2d_f32(x[b], ws[pq])
+        assert_close_f32(y_al[b], y_ref, s_ref, "image %d" % b)
+    y_un = run_2d(x, ws[pq], design, cuda_device, x_pitch=xp + 1, y_pitch=wd)
+    for b in range(batch):
+        y_ref, s_ref = oracle.conv2d_f32(x[b], ws[pq])
+        assert_close_f32(y_un[b], y_ref, s_ref, "image %d, unaligned rows" % b)
+    assert B.device_status() == 0
+
+
+@pytest.mark.parametrize("design", [B.OS, B.IS], ids=_ids)
+@pytest.mark.parametrize("pq", [(3, 3), (7, 7), (1, 1), (5, 13), (7, 15), (2, 4)], ids=lambda f: "%dx%d" % f)
+@pytest.mark.parametrize("size", [(1101, 83, 2), (3840, 140, 1), (1000, 41, 1), (4097, 64, 1), (64, 20, 3)],
+                         ids=lambda t: "%dx%dx%d" % t)
+def test_2d_u8_small_problems(cuda_device, design, pq, size):
+    wd, h, batch = size
+    p, q = pq
+    x, ws = inputs.gen_2d_u8s8(wd, h, [pq], seed=1400 + 16 * p + q + wd, batch=batch)
+    xp = (wd + 15) // 16 * 16
+    check_2d(x, ws[pq], design, cuda_device, x_pitch=xp)
+    check_2d(x, ws[pq], design, cuda_device, x_pitch=xp + 4, y_off=1)      # rows aligned to 4 bytes only, unaligned outputs
+    assert B.device_status() == 0
+
+
 # The fp32 OS / IS kernels for small filters (P*Q <= 25) have a form with eight PEs per lane that only large
 # problems reach (256-column strips x images x 8-row groups >= 4736); these cases are sized for it, with a ragged
 # right edge and a ragged last band.
