@@ -278,6 +278,43 @@ int sysconv_device_status(void);
  */
 int sysconv_selftest_wait_timeout(void *stream);
 
+/*
+ * Measured denominators for roofline figures (no counterpart in the paper, which reports only ratios to its
+ * own baseline; Section 6 explains its results by lane utilisation, which is what these rates normalise).
+ *
+ * sysconv_measure_peaks runs, on the current device, one block per SM that issues a long unrolled run of one
+ * kind of instruction and times itself with the SM's cycle counter, and a 128-bit streaming copy over the
+ * scratch buffer timed with CUDA events.  results_host[...] (at least SYSCONV_PEAK_COUNT doubles):
+ *   SYSCONV_PEAK_FFMA    fp32 fused multiply-adds per clock per SM
+ *   SYSCONV_PEAK_FFMA2   fp32 multiply-adds per clock per SM through the packed fp32x2 FMA, multiplicand (x, x)
+ *   SYSCONV_PEAK_IMAD    32-bit integer multiply-adds per clock per SM
+ *   SYSCONV_PEAK_DP4A    dp4a instructions per clock per SM (x 4 for 8-bit multiply-adds)
+ *   SYSCONV_PEAK_SHFL    warp-shuffle lane transfers per clock per SM
+ *   SYSCONV_PEAK_COPY_GBS  bytes read + written per second by the copy, in GB/s
+ *   SYSCONV_PEAK_SM_COUNT  SMs of the device
+ * scratch_dev: DEVICE memory owned by the caller, 256-byte aligned, at least 64 MiB (use several hundred MiB so
+ * that the copy is larger than the L2 cache); its contents are overwritten.  Synchronises the device; takes
+ * a few milliseconds.  SYSCONV_EINVAL for a null/small/misaligned buffer or count < SYSCONV_PEAK_COUNT.
+ *
+ * sysconv_floor_copy enqueues ONE plain streaming kernel on `stream`: widen == 0 copies bytes_in bytes from
+ * src_dev to dst_dev; widen == 1 reads bytes_in uint8 values and writes them as int32 (4 * bytes_in bytes).
+ * It moves the bytes of a convolution of that size and does none of its arithmetic: timed beside the
+ * convolution kernels it shows what a launch of that size costs at best.  Both pointers 16-byte aligned,
+ * bytes_in a multiple of 16, buffers must not overlap.
+ */
+enum {
+    SYSCONV_PEAK_FFMA = 0,
+    SYSCONV_PEAK_FFMA2 = 1,
+    SYSCONV_PEAK_IMAD = 2,
+    SYSCONV_PEAK_DP4A = 3,
+    SYSCONV_PEAK_SHFL = 4,
+    SYSCONV_PEAK_COPY_GBS = 5,
+    SYSCONV_PEAK_SM_COUNT = 6,
+    SYSCONV_PEAK_COUNT = 7
+};
+int sysconv_measure_peaks(void *scratch_dev, long long scratch_bytes, double *results_host, int count);
+int sysconv_floor_copy(const void *src_dev, void *dst_dev, long long bytes_in, int widen, void *stream);
+
 /* Library version, major*10000 + minor*100 + patch. */
 int sysconv_version(void);
 

@@ -83,6 +83,10 @@ def load_library():
     lib.sysconv_design_name.argtypes = [_c_int]
     lib.sysconv_version.restype = _c_int
     lib.sysconv_device_status.restype = _c_int
+    lib.sysconv_measure_peaks.restype = _c_int
+    lib.sysconv_measure_peaks.argtypes = [_vp, _c_ll, _vp, _c_int]
+    lib.sysconv_floor_copy.restype = _c_int
+    lib.sysconv_floor_copy.argtypes = [_vp, _vp, _c_ll, _c_int, _vp]
     lib.sysconv_selftest_wait_timeout.restype = _c_int
     lib.sysconv_selftest_wait_timeout.argtypes = [_vp]
     lib.sysconv_launch_count.restype = _c_ll
@@ -114,6 +118,29 @@ def selftest_wait_timeout(stream=None):
     st = int(load_library().sysconv_selftest_wait_timeout(_vp(_stream_ptr(stream))))
     if st != 0:
         raise SysconvError(st, "sysconv_selftest_wait_timeout")
+
+
+PEAK_NAMES = ("ffma_per_clk_sm", "ffma2_mac_per_clk_sm", "imad_per_clk_sm", "dp4a_per_clk_sm", "shfl_per_clk_sm",
+              "copy_gbs", "sm_count")
+
+
+def measure_peaks(scratch):
+    """Issue rates of the plain datapaths and the streaming-copy bandwidth of the current device, as a dict.
+    scratch: a CUDA uint8 tensor of at least 64 MiB (overwritten)."""
+    out = (ctypes.c_double * len(PEAK_NAMES))()
+    st = int(load_library().sysconv_measure_peaks(_vp(scratch.data_ptr()), scratch.numel() * scratch.element_size(),
+                                                   ctypes.cast(out, _vp), len(PEAK_NAMES)))
+    if st != 0:
+        raise SysconvError(st, "sysconv_measure_peaks")
+    return dict(zip(PEAK_NAMES, [float(v) for v in out]))
+
+
+def floor_copy(src, dst, bytes_in, widen=False, stream=None):
+    """One plain streaming kernel that moves the bytes of a convolution of that size (see sysconv.h)."""
+    st = int(load_library().sysconv_floor_copy(_vp(src.data_ptr()), _vp(dst.data_ptr()), int(bytes_in), 1 if widen else 0,
+                                                _vp(_stream_ptr(stream))))
+    if st != 0:
+        raise SysconvError(st, "sysconv_floor_copy")
 
 
 def launch_count():

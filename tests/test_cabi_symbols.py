@@ -152,3 +152,16 @@ def test_size_queries_reject_products_beyond_the_index_type(lib):
                                    vp(0))
     assert st == 1
     assert b.launch_count() == before
+
+
+def test_peak_measurement_argument_validation_needs_no_gpu(lib):
+    vp = ctypes.c_void_p
+    out = (ctypes.c_double * 8)()
+    assert lib.sysconv_measure_peaks(vp(0), ctypes.c_longlong(1 << 30), ctypes.cast(out, vp), 8) == 1          # null scratch
+    assert lib.sysconv_measure_peaks(vp(0x7f0000000000), ctypes.c_longlong(1 << 20), ctypes.cast(out, vp), 8) == 1   # too small
+    assert lib.sysconv_measure_peaks(vp(0x7f0000000010), ctypes.c_longlong(1 << 30), ctypes.cast(out, vp), 8) == 1   # misaligned
+    assert lib.sysconv_measure_peaks(vp(0x7f0000000000), ctypes.c_longlong(1 << 30), ctypes.cast(out, vp), 3) == 1   # too few results
+    assert lib.sysconv_floor_copy(vp(0), vp(0x7f0000000000), ctypes.c_longlong(1024), 0, vp(0)) == 1
+    assert lib.sysconv_floor_copy(vp(0x7f0000000000), vp(0x7f0000100000), ctypes.c_longlong(1000), 0, vp(0)) == 1    # not x16
+    assert lib.sysconv_floor_copy(vp(0x7f0000000004), vp(0x7f0000100000), ctypes.c_longlong(1024), 0, vp(0)) == 1    # misaligned
+    assert lib.sysconv_floor_copy(vp(0x7f0000000000), vp(0x7f0000100000), ctypes.c_longlong(1024), 2, vp(0)) == 1    # widen flag

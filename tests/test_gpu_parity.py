@@ -819,6 +819,31 @@ def test_host_multi_entry_point(cuda_device):
     assert B.device_status() == 0
 
 
+# ------------------------------------------------------------------------ measured peaks and yardstick kernels
+
+
+def test_measured_peaks_are_plausible_and_floor_kernels_move_the_bytes(cuda_device):
+    scratch = torch.empty(512 << 20, dtype=torch.uint8, device=cuda_device)
+    pk = B.measure_peaks(scratch)
+    assert pk["sm_count"] == torch.cuda.get_device_properties(cuda_device).multi_processor_count
+    # an SM has 128 fp32 lanes; nothing can exceed them and a healthy device gets most of the way there
+    assert 90 <= pk["ffma_per_clk_sm"] <= 129
+    assert 90 <= pk["ffma2_mac_per_clk_sm"] <= 257
+    assert 30 <= pk["imad_per_clk_sm"] <= 129
+    assert 30 <= pk["dp4a_per_clk_sm"] <= 129
+    assert 16 <= pk["shfl_per_clk_sm"] <= 129
+    assert 2000 <= pk["copy_gbs"] <= 9000
+    del scratch
+    src = torch.randint(0, 256, (1 << 20,), dtype=torch.uint8, device=cuda_device)
+    dst = torch.zeros(1 << 20, dtype=torch.uint8, device=cuda_device)
+    B.floor_copy(src, dst, src.numel())
+    wide = torch.full((1 << 20,), -1, dtype=torch.int32, device=cuda_device)
+    B.floor_copy(src, wide, src.numel(), widen=True)
+    torch.cuda.synchronize()
+    assert torch.equal(src, dst)
+    assert torch.equal(src.to(torch.int32), wide)
+
+
 # ------------------------------------------------------------------------ bounded device-side waits
 
 
