@@ -1,6 +1,6 @@
-"""ctypes front-end of ``conv_oracle.c`` (TEST INFRASTRUCTURE ONLY).
+"""ctypes front-end of ``conv_oracle.c`` and ``stencil_oracle.c`` (TEST INFRASTRUCTURE ONLY).
 
-Compiles the C file with gcc on first use (``-O2 -fopenmp``) into
+Compiles the C files with gcc on first use (``-O2 -fopenmp``) into
 ``oracle/_build/liboracle.so`` and exposes numpy-in / numpy-out functions.
 Argument checking and array allocation only; every sum is formed in the C file.
 """
@@ -12,7 +12,7 @@ import threading
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SRC = os.path.join(_HERE, "conv_oracle.c")
+_SRCS = [os.path.join(_HERE, "conv_oracle.c"), os.path.join(_HERE, "stencil_oracle.c")]
 _OUT_DIR = os.path.join(_HERE, "_build")
 _LIB_PATH = os.path.join(_OUT_DIR, "liboracle.so")
 _lock = threading.Lock()
@@ -27,11 +27,11 @@ def build_oracle(force: bool = False) -> str:
     """Compile the C oracle if the shared object is missing or stale."""
     os.makedirs(_OUT_DIR, exist_ok=True)
     stale = (not os.path.exists(_LIB_PATH)
-             or os.path.getmtime(_LIB_PATH) < os.path.getmtime(_SRC))
+             or os.path.getmtime(_LIB_PATH) < max(os.path.getmtime(p) for p in _SRCS))
     if force or stale:
         tmp = _LIB_PATH + ".tmp.%d" % os.getpid()
         cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11",
-               "-o", tmp, _SRC, "-lm"]
+               "-o", tmp] + _SRCS + ["-lm"]
         subprocess.run(cmd, check=True)
         os.replace(tmp, _LIB_PATH)
     return _LIB_PATH
@@ -61,6 +61,8 @@ def _load():
                                                    _vp, _c_ll]
             lib.oracle_conv2d_u8s8_i64.argtypes = [_vp, _c_int, _c_int, _c_ll, _vp, _c_int, _c_int,
                                                    _vp, _c_ll]
+            lib.oracle_stencil2d_f32.argtypes = [_vp, _c_int, _c_int, _c_ll, _vp, _c_int, _vp, _vp]
+            lib.oracle_stencil2d_f32.restype = _c_int
             for name in ("oracle_set_num_threads", "oracle_conv1d_f32",
                          "oracle_conv1d_f32_taps_outer", "oracle_conv1d_f32_at",
                          "oracle_conv2d_f32", "oracle_conv2d_f32_taps_outer",
@@ -239,3 +241,21 @@ def conv2d_u8s8_i64(x, w):
     y = np.empty((h - p + 1, wd - q + 1), dtype=np.int64)
     _load().oracle_conv2d_u8s8_i64(_ptr(x), wd, h, wd, _ptr(w), q, p, _ptr(y), wd - q + 1)
     return y
+
+
+def stencil2d_f32(u, k, sweeps, want_scale=True):
+    """``sweeps`` Jacobi sweeps of the 3x3 stencil k (k[dr+1][dc+1]) over the grid u with its outermost ring held
+    fixed, in fp64.  Returns (y, S): S = the same sweeps of |k| over |u| (the tolerance scale), or None."""
+    u = _as(u, np.float32, 2)
+    k = _as(k, np.float32, 2)
+    if k.shape != (3, 3):
+        raise ValueError("the stencil is 3 x 3")
+    if sweeps < 0:
+        raise ValueError("sweeps >= 0")
+    h, w = u.shape
+    y = np.empty((h, w), dtype=np.float64)
+    s = np.empty((h, w), dtype=np.float64) if want_scale else None
+    rc = _load().oracle_stencil2d_f32(_ptr(u), w, h, w, _ptr(k), int(sweeps), _ptr(y), _ptr(s) if want_scale else None)
+    if rc != 0:
+        raise MemoryError("oracle_stencil2d_f32")
+    return y, s
