@@ -275,6 +275,20 @@ def build_strided_cases(device):
         cases.append(Case("5/separable", "%d+%d" % (k, k), B.OS,
                           [checked(B.sysconv2d_separable, x2.data_ptr(), wd, h, wd, h * wd, u, v, yd.data_ptr(), y_pitch,
                                    oh * y_pitch, batch)], n_out, x.size * 4 + 4 * n_out, n_out * 2 * k))
+    # the second workload: Jacobi sweeps of a 3x3 stencil over the same 16 grids, up to four sweeps fused per pass
+    # (algorithmic bytes: the grid read and written once per pass of up to four sweeps)
+    five = np.array([[0, 0.125, 0], [0.125, 0.5, 0.125], [0, 0.125, 0]], np.float32)
+    nine = np.array([[0.0625, 0.125, 0.0625], [0.125, 0.25, 0.125], [0.0625, 0.125, 0.0625]], np.float32)
+    out = torch.empty((batch, h, wd), dtype=torch.float32, device=device)
+    scratch = torch.empty((batch, h, wd), dtype=torch.float32, device=device)
+    keep += [five, nine, out, scratch]
+    for name, k in (("5pt", five), ("9pt", nine)):
+        for sweeps in (1, 4, 8):
+            passes = -(-sweeps // 4)
+            cases.append(Case("5/stencil", "%s x%d" % (name, sweeps), B.OS,
+                              [checked(B.sysstencil2d, x2.data_ptr(), wd, h, wd, h * wd, k, sweeps, out.data_ptr(), wd, h * wd,
+                                       batch, scratch.data_ptr())], batch * h * wd * sweeps, 8 * x.size * passes,
+                              batch * (h - 2) * (wd - 2) * sweeps * (5 if name == "5pt" else 9)))
     return cases, keep
 
 

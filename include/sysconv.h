@@ -150,6 +150,33 @@ int sysconv2d_separable(const void *x_dev, int width, int height, long long x_pi
                         void *y_dev, long long y_pitch, long long y_batch_stride, int batch, void *stream);
 
 /*
+ * Iterated 3x3 stencil, a second workload on the same folded array (Section 1 of the paper names stencils
+ * beside convolution as what systolic arrays on GPUs are for; it evaluates none).
+ *
+ *   one sweep:  v[r][c] = sum_{dr,dc in {-1,0,1}} k[dr+1][dc+1] * u[r+dr][c+dc]   for 0 < r < height-1, 0 < c < width-1
+ *               v[r][c] = u[r][c]                                                  on the outermost ring (fixed values)
+ *   out = the sweep applied `sweeps` times (Jacobi iteration: every sweep reads only the previous sweep's grid).
+ *
+ * Columns are the PE dimension, inputs are forwarded between neighbouring PEs by shuffles as in the
+ * output-stationary convolution, and up to four sweeps are fused in one pass over the grid (time levels kept in
+ * PE registers), so the grid is read and written once per four sweeps.  Intermediate levels are rounded to fp32.
+ *   u_dev, out_dev   DEVICE pointers, fp32, `batch` grids of height x width, rows pitch / out_pitch elements
+ *                    apart, grids batch_stride / out_batch_stride elements apart (ignored when batch == 1)
+ *   k_host           HOST pointer to the nine coefficients, row-major k[dr+1][dc+1]; with all four corner
+ *                    coefficients zero (five-point stencil) their multiply-adds are skipped
+ *   sweeps           >= 1.  More than four sweeps run as a chain of launches whose intermediate grids alternate
+ *                    between out_dev and scratch_dev.
+ *   scratch_dev      DEVICE buffer with the size and layout of the output; needed only when sweeps > 4 (may be NULL
+ *                    otherwise); its contents are overwritten
+ * u and out (and scratch) must not overlap.  batch <= 65535 (SYSCONV_EUNSUPPORTED beyond).  Grids with fewer than
+ * three rows or columns have no interior: the output is a copy of the input.
+ */
+int sysstencil2d(const void *u_dev, int width, int height, long long pitch, long long batch_stride,
+                 const void *k_host, int sweeps,
+                 void *out_dev, long long out_pitch, long long out_batch_stride, int batch,
+                 void *scratch_dev, void *stream);
+
+/*
  * Generic space-time-transform executor (Sections 2.1-2.2 and the generic code pattern of Section 4).
  * The 1-D convolution UREs over the iteration space (c, q) are mapped by PE = p_c*c + p_q*q and
  * time = s_c*c + s_q*q; the dependences, delays and PE distances are derived from (P, s) alone, so the six

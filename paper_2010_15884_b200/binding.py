@@ -57,6 +57,8 @@ def load_library():
     lib.sysconv2d_separable.restype = _c_int
     lib.sysconv2d_separable.argtypes = [_vp, _c_int, _c_int, _c_ll, _c_ll, _vp, _c_int, _vp, _c_int, _vp, _c_ll, _c_ll,
                                         _c_int, _vp]
+    lib.sysstencil2d.restype = _c_int
+    lib.sysstencil2d.argtypes = [_vp, _c_int, _c_int, _c_ll, _c_ll, _vp, _c_int, _vp, _c_ll, _c_ll, _c_int, _vp, _vp]
     lib.sysconv_spacetime_describe.restype = _c_int
     lib.sysconv_spacetime_describe.argtypes = [_c_int, _c_int, _c_int, _c_int, _c_int, _vp, _vp]
     lib.sysconv1d_spacetime.restype = _c_int
@@ -381,6 +383,47 @@ def conv1d(x, w, design=OS, out=None, stream=None, stride=1):
     if st != 0:
         raise SysconvError(st, "sysconv1d" if stride == 1 else "sysconv1d_strided")
     return out.squeeze(0) if (squeeze and out.dim() == 2) else out
+
+
+def sysstencil2d(u_ptr, width, height, pitch, batch_stride, k_host, sweeps, out_ptr, out_pitch, out_batch_stride, batch,
+                 scratch_ptr, stream_ptr):
+    """Raw call (pointers are integers, k_host a numpy array of nine floats). Returns the status."""
+    k = np.ascontiguousarray(k_host, dtype=np.float32)
+    return int(load_library().sysstencil2d(_vp(u_ptr), int(width), int(height), int(pitch), int(batch_stride),
+                                            _vp(k.ctypes.data), int(sweeps), _vp(out_ptr), int(out_pitch),
+                                            int(out_batch_stride), int(batch), _vp(scratch_ptr), _vp(stream_ptr)))
+
+
+def stencil2d(u, k, sweeps, out=None, scratch=None, stream=None):
+    """`sweeps` Jacobi sweeps of the 3x3 stencil k over u (CUDA fp32, (h, w) or (batch, h, w), contiguous rows), the
+    outermost ring of every grid held fixed.  A scratch tensor like the output is allocated when sweeps > 4 and none
+    is given."""
+    import torch
+    if not u.is_cuda:
+        raise SysconvError(-1, "stencil2d (u is not a CUDA tensor; there is no CPU path)")
+    if u.dtype != torch.float32:
+        raise ValueError("stencil2d works on float32 grids")
+    squeeze = u.dim() == 2
+    u3 = u.unsqueeze(0) if squeeze else u
+    if u3.dim() != 3 or u3.stride(2) != 1:
+        raise ValueError("u must be (h, w) or (batch, h, w) with contiguous rows")
+    k = np.ascontiguousarray(k.detach().cpu().numpy() if hasattr(k, "detach") else k, dtype=np.float32)
+    if k.shape != (3, 3):
+        raise ValueError("the stencil is 3 x 3")
+    batch, h, wd = u3.shape
+    if out is None:
+        out = torch.empty((batch, h, wd), dtype=torch.float32, device=u.device)
+        o3 = out
+    else:
+        o3 = out.unsqueeze(0) if out.dim() == 2 else out
+    if sweeps > 4 and scratch is None:
+        scratch = torch.empty_strided(o3.shape, o3.stride(), dtype=torch.float32, device=u.device)
+    st = sysstencil2d(u3.data_ptr(), wd, h, u3.stride(1), u3.stride(0) if batch > 1 else 0, k, sweeps, o3.data_ptr(),
+                      o3.stride(1), o3.stride(0) if batch > 1 else 0, batch,
+                      scratch.data_ptr() if scratch is not None else 0, _stream_ptr(stream))
+    if st != 0:
+        raise SysconvError(st, "sysstencil2d")
+    return out.squeeze(0) if (squeeze and out.dim() == 3) else out
 
 
 def conv2d(x, w, design=OS, out=None, stream=None, stride=1):

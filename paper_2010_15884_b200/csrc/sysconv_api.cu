@@ -328,6 +328,51 @@ int sysconv2d_separable(const void *x_dev, int width, int height, long long x_pi
     return finish(err, launches);
 }
 
+int sysstencil2d(const void *u_dev, int width, int height, long long pitch, long long batch_stride, const void *k_host,
+                 int sweeps, void *out_dev, long long out_pitch, long long out_batch_stride, int batch, void *scratch_dev,
+                 void *stream)
+{
+    using namespace sysconv;
+    constexpr int kFused = 4;                   // sweeps fused in one launch
+    if (!u_dev || !out_dev || !k_host) return SYSCONV_EINVAL;
+    if (width < 1 || height < 1 || batch < 1 || sweeps < 1) return SYSCONV_EINVAL;
+    if (pitch < width || out_pitch < width) return SYSCONV_EINVAL;
+    const long long u_img = (long long)(height - 1) * pitch + width;
+    const long long o_img = (long long)(height - 1) * out_pitch + width;
+    if (batch > 1 && (batch_stride < u_img || out_batch_stride < o_img)) return SYSCONV_EINVAL;
+    if (batch == 1) { batch_stride = u_img; out_batch_stride = o_img; }
+    const unsigned long long u_bytes = ((unsigned long long)(batch - 1) * batch_stride + u_img) * 4ull;
+    const unsigned long long o_bytes = ((unsigned long long)(batch - 1) * out_batch_stride + o_img) * 4ull;
+    if (overlaps(u_dev, u_bytes, out_dev, o_bytes)) return SYSCONV_EINVAL;
+    const int launches_needed = (sweeps + kFused - 1) / kFused;
+    if (launches_needed > 1) {
+        if (!scratch_dev) return SYSCONV_EINVAL;
+        if (overlaps(scratch_dev, o_bytes, out_dev, o_bytes) || overlaps(scratch_dev, o_bytes, u_dev, u_bytes)) return SYSCONV_EINVAL;
+    }
+    if (batch > 65535) return SYSCONV_EUNSUPPORTED;
+    // Chain of launches, each fusing up to four sweeps; the intermediate grids alternate between the scratch
+    // buffer and the output (both in the output's layout) so that the last launch writes the output.
+    const float *k = static_cast<const float *>(k_host);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    Conv2DArgs a;
+    a.width = width; a.height = height; a.out_w = width; a.out_h = height; a.batch = batch;
+    const void *src = u_dev;
+    long long src_pitch = pitch, src_bstride = batch_stride;
+    int launches = 0, left = sweeps;
+    for (int l = 0; l < launches_needed; ++l) {
+        const int fused = left < kFused ? left : kFused;
+        void *dst = ((launches_needed - 1 - l) % 2 == 0) ? out_dev : scratch_dev;
+        a.x = src; a.y = dst;
+        a.x_pitch = src_pitch; a.x_bstride = src_bstride;
+        a.y_pitch = out_pitch; a.y_bstride = out_batch_stride;
+        const cudaError_t err = launch_stencil2d_f32(a, k, fused, s, &launches);
+        if (err != cudaSuccess) return finish(err, launches);
+        src = dst; src_pitch = out_pitch; src_bstride = out_batch_stride;
+        left -= fused;
+    }
+    return finish(cudaSuccess, launches);
+}
+
 int sysconv_spacetime_describe(int p_c, int p_q, int s_c, int s_q, int q, int *info, char *name)
 {
     return sysconv::spacetime_describe(p_c, p_q, s_c, s_q, q, info, name);

@@ -93,6 +93,9 @@ cudaError_t launch_conv2d_f32_stride2(int design, const Conv2DArgs &a, const flo
 cudaError_t launch_conv2d_f32_separable(const Conv2DArgs &a, const float *u, int p, const float *v, int q, cudaStream_t s,
                                         int *launches);
 
+// iterated 3x3 stencil (stencil2d_f32.cu): `fused` sweeps (1..4) in one launch; a.out_w/out_h unused (output = grid size)
+cudaError_t launch_stencil2d_f32(const Conv2DArgs &a, const float *k9, int fused, cudaStream_t s, int *launches);
+
 // generic space-time executor (spacetime.cu): *status receives the planning result
 int spacetime_describe(int pc, int pq, int sc, int sq, int q, int *out10, char *name4);
 cudaError_t launch_spacetime_conv1d(const float *x, long long n, const float *w, int q, float *y, int pc, int pq, int sc,

@@ -165,3 +165,18 @@ def test_peak_measurement_argument_validation_needs_no_gpu(lib):
     assert lib.sysconv_floor_copy(vp(0x7f0000000000), vp(0x7f0000100000), ctypes.c_longlong(1000), 0, vp(0)) == 1    # not x16
     assert lib.sysconv_floor_copy(vp(0x7f0000000004), vp(0x7f0000100000), ctypes.c_longlong(1024), 0, vp(0)) == 1    # misaligned
     assert lib.sysconv_floor_copy(vp(0x7f0000000000), vp(0x7f0000100000), ctypes.c_longlong(1024), 2, vp(0)) == 1    # widen flag
+
+
+def test_stencil_argument_validation_needs_no_gpu(lib):
+    import numpy as np
+    from paper_2010_15884_b200 import binding as b
+    k = np.ones((3, 3), np.float32)
+    u, o, sc = 0x10000, 0x90000000, 0xa0000000
+    assert b.sysstencil2d(0, 64, 64, 64, 0, k, 1, o, 64, 0, 1, 0, 0) == 1          # null grid
+    assert b.sysstencil2d(u, 64, 64, 63, 0, k, 1, o, 64, 0, 1, 0, 0) == 1          # pitch < width
+    assert b.sysstencil2d(u, 64, 64, 64, 0, k, 0, o, 64, 0, 1, 0, 0) == 1          # no sweeps
+    assert b.sysstencil2d(u, 64, 64, 64, 0, k, 1, u + 64, 64, 0, 1, 0, 0) == 1     # output overlaps the input
+    assert b.sysstencil2d(u, 64, 64, 64, 0, k, 5, o, 64, 0, 1, 0, 0) == 1          # five sweeps need a scratch buffer
+    assert b.sysstencil2d(u, 64, 64, 64, 0, k, 5, o, 64, 0, 1, o + 128, 0) == 1    # scratch overlaps the output
+    assert b.sysstencil2d(u, 64, 64, 64, 64 * 64, k, 2, o, 64, 64 * 63, 2, sc, 0) == 1    # output batch stride too small
+    assert b.sysstencil2d(u, 8, 8, 8, 64, k, 2, o, 8, 64, 70000, sc, 0) == 2       # batch beyond 65535

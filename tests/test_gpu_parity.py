@@ -732,6 +732,120 @@ def test_separable_full_size_sampled(cuda_device):
     assert_close_f32(y[1].cpu().numpy()[rows, cols], y_ref, s_ref, "sampled")
 
 
+# ------------------------------------------------------------------------ iterated 3x3 stencil (second workload)
+
+K_FIVE = np.array([[0, 0.2, 0], [0.15, 0.3, 0.25], [0, 0.1, 0]], np.float32)
+K_NINE = np.array([[0.05, 0.2, -0.1], [0.15, 0.3, 0.25], [0.07, 0.1, -0.02]], np.float32)
+
+
+def check_stencil(u_np, k, sweeps, device, pitch=None, out_pitch=None, u_off=0, o_off=0):
+    """u_np: (batch, h, w).  Runs sysstencil2d through the C ABI, checks canaries, compares every point of every
+    grid with the oracle: |y - y_ref| <= 1e-5 * S, S = the same sweeps of |k| over |u|."""
+    batch, h, wd = u_np.shape
+    pitch = pitch or wd
+    out_pitch = out_pitch or wd
+    ub = torch.zeros(u_off + batch * h * pitch + 16, dtype=torch.float32, device=device)
+    ob = torch.full((o_off + batch * h * out_pitch + 64,), CANARY, dtype=torch.float32, device=device)
+    sb = torch.full((o_off + batch * h * out_pitch + 64,), CANARY, dtype=torch.float32, device=device)
+    ub[u_off: u_off + batch * h * pitch].view(batch, h, pitch)[:, :, :wd] = torch.from_numpy(u_np).to(device)
+    st = B.sysstencil2d(ub.data_ptr() + 4 * u_off, wd, h, pitch, h * pitch, k, sweeps, ob.data_ptr() + 4 * o_off, out_pitch,
+                        h * out_pitch, batch, sb.data_ptr() + 4 * o_off if sweeps > 4 else 0,
+                        torch.cuda.current_stream().cuda_stream)
+    assert st == 0, B.status_string(st)
+    torch.cuda.synchronize()
+    for buf in (ob, sb):
+        yh = buf.cpu().numpy()
+        body = yh[o_off: o_off + batch * h * out_pitch].reshape(batch, h, out_pitch)
+        assert (body[:, :, wd:] == CANARY).all(), "write into the pitch padding"
+        assert (yh[:o_off] == CANARY).all() and (yh[o_off + batch * h * out_pitch:] == CANARY).all()
+    yh = ob.cpu().numpy()
+    body = yh[o_off: o_off + batch * h * out_pitch].reshape(batch, h, out_pitch)
+    for b in range(batch):
+        y_ref, s_ref = oracle.stencil2d_f32(u_np[b], k, sweeps)
+        assert_close_f32(body[b, :, :wd], y_ref, s_ref, "grid %d, %d sweeps" % (b, sweeps))
+
+
+@pytest.mark.parametrize("k", [K_FIVE, K_NINE], ids=["five_point", "nine_point"])
+@pytest.mark.parametrize("sweeps", [1, 2, 3, 4, 5, 7, 8, 9, 13])
+def test_stencil_sweep_counts(cuda_device, k, sweeps):
+    rng = np.random.default_rng(1500 + sweeps)
+    u = rng.uniform(-1, 1, (2, 150, 300)).astype(np.float32)
+    check_stencil(u, k, sweeps, cuda_device)
+
+
+@pytest.mark.parametrize("sweeps", [1, 3, 4, 6])
+@pytest.mark.parametrize("hw", [(1, 1), (1, 9), (9, 1), (2, 2), (3, 3), (3, 200), (200, 3), (4, 5), (17, 119), (18, 120),
+                                (19, 121), (40, 127), (41, 128), (42, 129), (130, 241), (131, 255), (260, 113)])
+def test_stencil_ragged_grid_sizes(cuda_device, sweeps, hw):
+    # grids without interior, widths around the 120- and 112-column strips, heights around the band edges
+    rng = np.random.default_rng(1600 + hw[0] + hw[1])
+    u = rng.uniform(0, 1, (1, hw[0], hw[1])).astype(np.float32)
+    check_stencil(u, K_NINE, sweeps, cuda_device)
+
+
+@pytest.mark.parametrize("layout", [(203, 201, 1, 3), (204, 204, 0, 0), (208, 200, 4, 4), (201, 202, 2, 2)])
+def test_stencil_pitches_and_alignment(cuda_device, layout):
+    pitch, out_pitch, u_off, o_off = layout
+    rng = np.random.default_rng(1700)
+    u = rng.uniform(-1, 1, (3, 70, 200)).astype(np.float32)
+    for sweeps in (2, 6):
+        check_stencil(u, K_FIVE, sweeps, cuda_device, pitch=pitch, out_pitch=out_pitch, u_off=u_off, o_off=o_off)
+
+
+def test_stencil_fixed_points_exact_integers_and_non_finite(cuda_device):
+    # a constant field under coefficients that sum to one (dyadic, exact) is a fixed point at every sweep count
+    k = np.array([[0.125, 0.0625, 0.0625], [0.25, 0.25, 0.0625], [0.0625, 0.0625, 0.0625]], np.float32)
+    u = torch.full((1, 300, 500), 3.0, device=cuda_device)
+    for sweeps in (1, 4, 11):
+        assert torch.equal(B.stencil2d(u, k, sweeps), u)
+    # integer data and dyadic coefficients: exact in fp32 whatever the order, so every bit must match the oracle
+    rng = np.random.default_rng(1800)
+    ui = rng.integers(-8, 9, (2, 140, 260)).astype(np.float32)
+    kd = np.array([[0.25, 0.5, 0.25], [0.5, -1.0, 0.5], [0.25, 0.5, 0.25]], np.float32)
+    for sweeps in (1, 4, 6):
+        y = B.stencil2d(torch.from_numpy(ui).to(cuda_device), kd, sweeps).cpu().numpy()
+        for b in range(2):
+            np.testing.assert_array_equal(y[b].astype(np.float64), oracle.stencil2d_f32(ui[b], kd, sweeps)[0])
+    # a non-finite value spreads exactly as the definition says: one ring of neighbours per sweep, never through
+    # the fixed boundary ring
+    uf = rng.uniform(0, 1, (1, 90, 260)).astype(np.float32)
+    for r, c, v in ((0, 0, np.nan), (40, 127, np.inf), (41, 128, -np.inf), (89, 130, np.nan), (30, 0, np.inf), (60, 259, np.nan)):
+        uf[0, r, c] = v
+    for sweeps in (1, 3, 4, 5):
+        with np.errstate(invalid="ignore"):
+            y_ref, s_ref = oracle.stencil2d_f32(uf[0], K_NINE, sweeps)
+        y = B.stencil2d(torch.from_numpy(uf).to(cuda_device), K_NINE, sweeps).cpu().numpy()[0].astype(np.float64)
+        _assert_same_where_finite(y, y_ref, s_ref, "%d sweeps" % sweeps)
+
+
+def test_stencil_many_small_grids_and_the_eigenfunction(cuda_device):
+    rng = np.random.default_rng(1900)
+    check_stencil(rng.uniform(-1, 1, (40, 33, 47)).astype(np.float32), K_NINE, 4, cuda_device)
+    # Dirichlet eigenfunction of the five-point Jacobi sweep: decays by its closed-form factor per sweep
+    h, w, a = 129, 257, 0.125
+    r, c = np.mgrid[0:h, 0:w]
+    u = (np.sin(np.pi * r / (h - 1)) * np.sin(np.pi * c / (w - 1))).astype(np.float32)
+    u[0] = u[-1] = 0
+    u[:, 0] = u[:, -1] = 0
+    k = np.array([[0, a, 0], [a, 1 - 4 * a, a], [0, a, 0]], np.float32)
+    lam = 1 - 4 * a + 2 * a * (np.cos(np.pi / (h - 1)) + np.cos(np.pi / (w - 1)))
+    y = B.stencil2d(torch.from_numpy(u).to(cuda_device), k, 16).cpu().numpy().astype(np.float64)
+    np.testing.assert_allclose(y, lam ** 16 * u.astype(np.float64), rtol=0, atol=5e-6)
+
+
+@pytest.mark.parametrize("sweeps", [1, 4, 8])
+def test_stencil_full_size_every_point(cuda_device, sweeps):
+    """16 x 4096 x 4096, the launch configuration bench.py times: every point of every grid against the oracle."""
+    x, _ = inputs.make_config(5, scale=dict(filters=[3]))
+    xd = torch.from_numpy(x).to(cuda_device)
+    y = B.stencil2d(xd, K_NINE if sweeps != 4 else K_FIVE, sweeps)
+    torch.cuda.synchronize()
+    del xd
+    for b in range(16):
+        y_ref, s_ref = oracle.stencil2d_f32(x[b], K_NINE if sweeps != 4 else K_FIVE, sweeps)
+        assert_close_f32(y[b].cpu().numpy(), y_ref, s_ref, "grid %d" % b)
+
+
 # ------------------------------------------------------------------------ generic space-time executor
 
 ST_PAPER = {"SBM": ((1, 1), (0, 1)), "BSM": ((0, 1), (1, 1)), "FSM": ((0, 1), (1, -1)), "BFS": ((1, 0), (1, 1)),
