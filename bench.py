@@ -661,7 +661,7 @@ def run_ours(args):
             line["detail"] = all_config_detail(device, hbm_gbs, peak_kind, sm_max, skip=cfg_id,
                                                reps=args.detail_reps)
             line["target"] = target_table(mine + line["detail"], (1, 2, 3, 4, 5))
-            line["six_designs_n2p24"] = six_designs_table(device, args.detail_reps)
+            line["six_designs_paper_experiment"] = six_designs_table(device, args.detail_reps, hbm_gbs)
             line["cfg1_step_in_cuda_graph"] = graph_replay_ms(1, device, 200)
         print(json.dumps(line))
     if world > 1:
@@ -801,26 +801,32 @@ def graph_replay_ms(cfg_id, device, reps):
     return out
 
 
-def six_designs_table(device, reps):
-    """The shape of the paper's Table 3 / Table 4 experiment on B200: the six 1-D designs at filter sizes 2 and 5,
-    throughput relative to FBS (the paper compared with the GEN9.5 sampler, which does not exist here), beside the
-    analytical model's outturn and lane utilisation for 16 outputs, filter size 5 (Table 4)."""
+def six_designs_table(device, reps, hbm_gbs):
+    """The paper's own experiment (Section 6, Tables 3 and 4) on B200: more than ten million independent 1-D
+    convolutions of 16 outputs each, filter sizes 2 and 5, through all six designs (small unfolded arrays side by
+    side in a warp).  Throughput = outputs / kernel time, as in the paper; beside it the analytical model's outturn
+    and lane utilisation for 16 outputs, filter size 5 (Table 4), and the paper's own relative performance against
+    the GEN9.5 sampler (Table 3; context only: that baseline does not exist here)."""
     import torch
     from paper_2010_15884_b200 import binding as B
     from paper_2010_15884_b200 import inputs
     model = {"SBM": (3.2, 80), "BSM": (0.8, 80), "FSM": (0.8, 80), "BFS": (0.8, 25), "FFS": (0.46, 14), "FBS": (3.2, 100)}
+    paper_rel = {"SBM": (157, 147), "BSM": (67, 49), "FSM": (56, 39), "BFS": (56, 48), "FFS": (33, 30), "FBS": (159, 157)}
     enum = {"SBM": B.IS, "BSM": B.WS, "FSM": B.FSM, "BFS": B.BFS, "FFS": B.FFS, "FBS": B.OS}
-    n = 1 << 24
-    x, ws = inputs.gen_1d_f32(n, [2, 5], seed=5)
-    xd = torch.from_numpy(x).to(device)
+    tiles, c_out = 10 * (1 << 20), 16
     stream = torch.cuda.current_stream().cuda_stream
     rows = []
-    for q, w in ws.items():
-        yd = torch.empty(n - q + 1, dtype=torch.float32, device=device)
+    for qi, q in enumerate((2, 5)):
+        n = c_out + q - 1
+        x, ws = inputs.gen_1d_f32(tiles * n, [q], seed=60 + q)
+        xd = torch.from_numpy(x).to(device)
+        yd = torch.empty(tiles * c_out, dtype=torch.float32, device=device)
+        w = ws[q]
+        alg_bytes = 4.0 * tiles * (n + c_out)
         times = {}
         for name, d in enum.items():
-            def launch(d=d, w=w, q=q, yd=yd):
-                st = B.sysconv1d(xd.data_ptr(), n, n, w, q, yd.data_ptr(), n - q + 1, 1, B.F32, d, stream)
+            def launch(d=d):
+                st = B.sysconv1d(xd.data_ptr(), n, n, w, q, yd.data_ptr(), c_out, tiles, B.F32, d, stream)
                 if st != 0:
                     raise B.SysconvError(st, "sysconv1d")
             for _ in range(3):
@@ -831,27 +837,16 @@ def six_designs_table(device, reps):
                 e0.record(); launch(); e1.record(); e1.synchronize()
                 ts.append(e0.elapsed_time(e1))
             times[name] = statistics.median(ts)
-        # the same six designs through the generic space-time executor (one PE per lane, CheckTime, run-time (P; s))
-        from paper_2010_15884_b200 import designspace
-        generic = {}
-        for name, (P, s) in designspace.PAPER_DESIGNS.items():
-            def launch_g(P=P, s=s, w=w, q=q, yd=yd):
-                st = B.sysconv1d_spacetime(xd.data_ptr(), n, w, q, yd.data_ptr(), P, s, stream)
-                if st != 0:
-                    raise B.SysconvError(st, "sysconv1d_spacetime")
-            launch_g()
-            ts = []
-            for _ in range(max(3, reps // 4)):
-                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record(); launch_g(); e1.record(); e1.synchronize()
-                ts.append(e0.elapsed_time(e1))
-            generic[name] = statistics.median(ts)
         for name in enum:
-            rows.append({"design": name, "filter": q, "ms": round(times[name], 5),
-                         "generic_executor_ms": round(generic[name], 4),
-                         "gpix_s": round((n - q + 1) / (times[name] * 1e-3) / 1e9, 2),
+            rows.append({"design": name, "filter": q, "signals": tiles, "outputs_per_signal": c_out,
+                         "ms": round(times[name], 5),
+                         "gpix_s": round(tiles * c_out / (times[name] * 1e-3) / 1e9, 2),
+                         "hbm_frac": round(alg_bytes / (times[name] * 1e-3) / 1e9 / hbm_gbs, 4),
                          "relative_to_FBS": round(times["FBS"] / times[name], 3),
-                         "model_outturn_q5": model[name][0], "model_utilisation_pct_q5": model[name][1]})
+                         "model_outturn_q5": model[name][0], "model_utilisation_pct_q5": model[name][1],
+                         "paper_pct_of_gen9_sampler": paper_rel[name][qi]})
+        del xd, yd
+        torch.cuda.empty_cache()
     return rows
 
 

@@ -215,6 +215,8 @@ int sysconv1d(const void *x_dev, long long n, long long x_batch_stride, const vo
         a.x_bstride = x_batch_stride; a.y_bstride = y_batch_stride; a.batch = batch;
         const float *w = static_cast<const float *>(w_host);
         int launches = 0;
+        // a batch of tiny signals (the paper's own experiment shape): small arrays side by side in a warp
+        if (conv1d_tiles_eligible(a, design, q)) return finish(launch_conv1d_f32_tiles(design, a, w, q, s, &launches), launches);
         const DeviceInfo *d = device_info();
         if (!d) return SYSCONV_ECUDA;
         cudaError_t err = design == SYSCONV_OS   ? launch_conv1d_f32_os(a, w, q, d->status_word, s, &launches)

@@ -83,6 +83,10 @@ cudaError_t launch_conv1d_f32_ws(const Conv1DArgs &a, const float *w, int q, uns
 cudaError_t launch_conv1d_f32_other(int design, const Conv1DArgs &a, const float *w, int q, unsigned *status_word,
                                     cudaStream_t s, int *launches);
 
+// batches of tiny signals (at most 32 outputs, at most 8 taps): small unfolded arrays side by side in a warp, all six designs
+bool conv1d_tiles_eligible(const Conv1DArgs &a, int design, int q);
+cudaError_t launch_conv1d_f32_tiles(int design, const Conv1DArgs &a, const float *w, int q, cudaStream_t s, int *launches);
+
 // stride-2 forms (design = SYSCONV_OS or SYSCONV_IS); a.n_out / a.out_w, a.out_h are the strided output sizes
 cudaError_t launch_conv1d_f32_stride2(int design, const Conv1DArgs &a, const float *w, int q, unsigned *status_word,
                                       cudaStream_t s, int *launches);

@@ -183,6 +183,72 @@ def test_1d_many_tiles_batch(cuda_device, design):
     assert B.device_status() == 0
 
 
+# ---- batches of tiny signals: the paper's own experiment shape (Section 6), small unfolded arrays side by side
+ALL_DESIGNS = DESIGNS + OTHER_DESIGNS
+
+
+def tiles_reference(x2, w):
+    """Oracle for a batch of short signals in ONE call: laid end to end they form one long signal whose valid
+    convolution holds, at position b*n + c (c < n-q+1), exactly output c of signal b."""
+    batch, n = x2.shape
+    q = w.shape[0]
+    y, s = oracle.conv1d_f32(x2.reshape(-1), w)
+    idx = (np.arange(batch)[:, None] * n + np.arange(n - q + 1)[None, :])
+    return y[idx], s[idx]
+
+
+@pytest.mark.parametrize("design", ALL_DESIGNS, ids=_ids)
+@pytest.mark.parametrize("q", [1, 2, 5, 8])
+@pytest.mark.parametrize("c_out", [1, 2, 4, 15, 16, 17, 25, 32])
+def test_1d_tiny_signals_all_designs(cuda_device, design, q, c_out):
+    n = c_out + q - 1
+    rng = np.random.default_rng(2900 + 64 * q + c_out)
+    w = (rng.random(q, dtype=np.float32) * 2 - 1).astype(np.float32)
+    for batch, stride in ((2, None), (7, n + 3), (1000, None), (4099, n + 1)):
+        x = (rng.random((batch, n), dtype=np.float32) * 2 - 1).astype(np.float32)
+        y = run_1d(x, w, design, cuda_device, batch_stride=stride)
+        y_ref, s_ref = tiles_reference(x, w)
+        assert_close_f32(y, y_ref, s_ref, "%s q=%d C=%d batch=%d" % (_ids(design), q, c_out, batch))
+
+
+@pytest.mark.parametrize("design", ALL_DESIGNS, ids=_ids)
+def test_1d_tiny_signals_exact_integers_and_non_finite(cuda_device, design):
+    rng = np.random.default_rng(2950)
+    x = rng.integers(-50, 51, (3000, 20)).astype(np.float32)
+    w = rng.integers(-9, 10, 5).astype(np.float32)
+    y_ref, _ = tiles_reference(x, w)
+    np.testing.assert_array_equal(run_1d(x, w, design, cuda_device).astype(np.float64), y_ref)
+    xf = (rng.random((500, 20), dtype=np.float32) * 2 - 1).astype(np.float32)
+    xf[3, 0], xf[3, 19], xf[100, 7], xf[499, 15] = np.inf, np.nan, -np.inf, np.nan
+    wf = (rng.random(5, dtype=np.float32) * 2 - 1).astype(np.float32)
+    with np.errstate(invalid="ignore"):
+        refs = [oracle.conv1d_f32(row, wf) for row in xf]
+    y = run_1d(xf, wf, design, cuda_device)
+    _assert_same_where_finite(y, np.stack([r[0] for r in refs]), np.stack([r[1] for r in refs]), "non-finite")
+
+
+@pytest.mark.parametrize("q", [2, 5])
+def test_1d_paper_experiment_shape_full_size(cuda_device, q):
+    """More than ten million independent convolutions of 16 outputs each (Section 6), filter sizes 2 and 5, all six
+    designs: EVERY output against the oracle."""
+    tiles, c_out = 10 * (1 << 20), 16
+    n = c_out + q - 1
+    x, ws = inputs.gen_1d_f32(tiles * n, [q], seed=60 + q)
+    x = x.reshape(tiles, n)
+    y_ref, s_ref = tiles_reference(x, ws[q])
+    xd = torch.from_numpy(x).to(cuda_device)
+    yd = torch.empty((tiles, c_out), dtype=torch.float32, device=cuda_device)
+    for design in ALL_DESIGNS:
+        yd.fill_(CANARY)
+        B.conv1d(xd, ws[q], design, out=yd)
+        torch.cuda.synchronize()
+        y = yd.cpu().numpy()
+        for lo in range(0, tiles, 1 << 21):
+            assert_close_f32(y[lo:lo + (1 << 21)], y_ref[lo:lo + (1 << 21)], s_ref[lo:lo + (1 << 21)],
+                             "%s q=%d tiles %d.." % (_ids(design), q, lo))
+    assert B.device_status() == 0
+
+
 @pytest.mark.parametrize("design", OTHER_DESIGNS, ids=_ids)
 @pytest.mark.parametrize("q", [1, 2, 3, 5, 8, 13, 16, 17, 31, 32])
 def test_1d_other_designs_filter_lengths(cuda_device, design, q):
