@@ -122,9 +122,15 @@ int sysconv2d(const void *x_dev, int width, int height, long long x_pitch, long 
  * FBS design of Table 2), and y(r, c) = sum_p sum_q x(stride_r*r + p, stride_c*c + q) w(p, q) with
  * ((height-p)/stride_r + 1) x ((width-q)/stride_c + 1) outputs per image (Section 5 runs the strided
  * design row by row).  All other arguments as for sysconv1d / sysconv2d.
- * Stride 1 is the unstrided call.  Stride 2 (both directions in 2-D) is built for fp32 data, the
- * SYSCONV_OS and SYSCONV_IS designs, q <= 32 in 1-D and p, q <= 7 and batch <= 65535 in 2-D; every other combination returns
- * SYSCONV_EUNSUPPORTED (strides below 1: SYSCONV_EINVAL).
+ * Stride 1 is the unstrided call.  fp32 data only.
+ *   - stride 2 (both directions in 2-D), SYSCONV_OS and SYSCONV_IS, q <= 32 in 1-D, p, q <= 7 in 2-D: the
+ *     fully unrolled stride-2 arrays.
+ *   - any other strides (3, 4, ..., different strides per direction, stride 2 with larger filters up to
+ *     15 x 15), SYSCONV_OS only: the same output-stationary array with run-time strides -- the stride-2 cell's
+ *     X(c,q) = X(c+1, q-2) read as X(c+1, q-stride).  Slower than the unrolled kernels; 1-D signals need
+ *     n < 2^31 there.
+ *   batch <= 65535.  Every other combination (integer data, the weight-stationary design, SYSCONV_IS beyond the
+ *   first case, the designs FSM/BFS/FFS) returns SYSCONV_EUNSUPPORTED; strides below 1: SYSCONV_EINVAL.
  */
 int sysconv1d_strided(const void *x_dev, long long n, long long x_batch_stride,
                       const void *w_host, int q, int stride,

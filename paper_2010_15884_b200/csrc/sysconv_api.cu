@@ -254,7 +254,19 @@ int sysconv1d_strided(const void *x_dev, long long n, long long x_batch_stride, 
     const unsigned long long x_bytes = ((unsigned long long)(batch - 1) * x_batch_stride + n) * in_elt_bytes(dtype);
     const unsigned long long y_bytes = ((unsigned long long)(batch - 1) * y_batch_stride + n_out) * 4ull;
     if (overlaps(x_dev, x_bytes, y_dev, y_bytes)) return SYSCONV_EINVAL;
-    if (stride != 2 || dtype != SYSCONV_F32 || q > kMaxQ1) return SYSCONV_EUNSUPPORTED;
+    if (dtype != SYSCONV_F32 || q > kMaxQ1) return SYSCONV_EUNSUPPORTED;
+    if (stride != 2) {
+        // any other stride: the run-time-stride output-stationary array, the signals as one-row images
+        if (design != SYSCONV_OS || batch > 65535 || n > 0x7fffffffLL) return SYSCONV_EUNSUPPORTED;
+        Conv2DArgs g;
+        g.x = x_dev; g.y = y_dev;
+        g.width = static_cast<int>(n); g.height = 1; g.out_w = static_cast<int>(n_out); g.out_h = 1;
+        g.x_pitch = n; g.y_pitch = n_out; g.x_bstride = x_batch_stride; g.y_bstride = y_batch_stride; g.batch = batch;
+        int launches = 0;
+        const cudaError_t err = launch_conv_f32_strided_any(g, static_cast<const float *>(w_host), q, 1, stride, 1,
+                                                            static_cast<cudaStream_t>(stream), &launches);
+        return finish(err, launches);
+    }
     if (design != SYSCONV_OS && design != SYSCONV_IS) return SYSCONV_EUNSUPPORTED;
     Conv1DArgs a;
     a.x = x_dev; a.y = y_dev; a.n = n; a.n_out = n_out;
@@ -288,7 +300,7 @@ int sysconv2d_strided(const void *x_dev, int width, int height, long long x_pitc
     const unsigned long long x_bytes = ((unsigned long long)(batch - 1) * x_batch_stride + x_img) * in_elt_bytes(dtype);
     const unsigned long long y_bytes = ((unsigned long long)(batch - 1) * y_batch_stride + y_img) * 4ull;
     if (overlaps(x_dev, x_bytes, y_dev, y_bytes)) return SYSCONV_EINVAL;
-    if (stride_c != 2 || stride_r != 2 || dtype != SYSCONV_F32 || batch > 65535) return SYSCONV_EUNSUPPORTED;
+    if (dtype != SYSCONV_F32 || batch > 65535 || q > kMaxQ2 || p > kMaxP2) return SYSCONV_EUNSUPPORTED;
     if (design != SYSCONV_OS && design != SYSCONV_IS) return SYSCONV_EUNSUPPORTED;
     Conv2DArgs a;
     a.x = x_dev; a.y = y_dev;
@@ -296,8 +308,16 @@ int sysconv2d_strided(const void *x_dev, int width, int height, long long x_pitc
     a.x_pitch = x_pitch; a.y_pitch = y_pitch;
     a.x_bstride = x_batch_stride; a.y_bstride = y_batch_stride; a.batch = batch;
     int launches = 0;
-    const cudaError_t err = launch_conv2d_f32_stride2(design, a, static_cast<const float *>(w_host), q, p,
-                                                      static_cast<cudaStream_t>(stream), &launches);
+    cudaError_t err;
+    if (stride_c == 2 && stride_r == 2 && p <= 7 && q <= 7) {
+        err = launch_conv2d_f32_stride2(design, a, static_cast<const float *>(w_host), q, p,
+                                        static_cast<cudaStream_t>(stream), &launches);
+    } else {
+        // other strides, mixed strides, larger filters: the run-time-stride output-stationary array
+        if (design != SYSCONV_OS) return SYSCONV_EUNSUPPORTED;
+        err = launch_conv_f32_strided_any(a, static_cast<const float *>(w_host), q, p, stride_c, stride_r,
+                                          static_cast<cudaStream_t>(stream), &launches);
+    }
     return finish(err, launches);
 }
 

@@ -93,6 +93,10 @@ cudaError_t launch_conv1d_f32_stride2(int design, const Conv1DArgs &a, const flo
 cudaError_t launch_conv2d_f32_stride2(int design, const Conv2DArgs &a, const float *w, int q, int p, cudaStream_t s,
                                       int *launches);
 
+// any strides, output-stationary design, fp32, up to 225 taps (conv_f32_strided_any.cu); 1-D = one row, p = 1
+cudaError_t launch_conv_f32_strided_any(const Conv2DArgs &a, const float *w, int q, int p, int sc, int sr, cudaStream_t s,
+                                        int *launches);
+
 // separable 2-D convolution (conv2d_f32_sep.cu): u = p vertical taps, v = q horizontal taps
 cudaError_t launch_conv2d_f32_separable(const Conv2DArgs &a, const float *u, int p, const float *v, int q, cudaStream_t s,
                                         int *launches);

@@ -87,16 +87,16 @@ def test_strided_argument_validation_needs_no_gpu(lib):
     assert b.sysconv1d_strided(0, 100, 100, w, 4, 2, y, 49, 1, b.F32, b.OS, 0) == 1        # null x
     assert b.sysconv1d_strided(x, 3, 3, w, 4, 2, y, 1, 1, b.F32, b.OS, 0) == 1             # n < q
     assert b.sysconv1d_strided(x, 100, 100, w, 4, 2, y, 40, 2, b.F32, b.OS, 0) == 1        # y batch stride < n_out
-    assert b.sysconv1d_strided(x, 100, 100, w, 4, 3, y, 33, 1, b.F32, b.OS, 0) == 2        # stride 3: not built
+    assert b.sysconv1d_strided(x, 100, 100, w, 4, 3, y, 33, 1, b.F32, b.IS, 0) == 2        # stride 3: output-stationary only
     assert b.sysconv1d_strided(x, 100, 100, w, 4, 2, y, 49, 1, b.F32, b.WS, 0) == 2        # WS: not built
     assert b.sysconv1d_strided(x, 100, 100, w, 4, 2, y, 49, 1, b.U8S8_S32, b.OS, 0) == 2   # integer: not built
     assert b.sysconv2d_strided(x, 64, 64, 64, 0, w2, 3, 3, 2, 0, y, 31, 0, 1, b.F32, b.OS, 0) == 1     # stride_r < 1
     assert b.sysconv2d_strided(x, 64, 64, 64, 0, w2, 3, 3, 2, 2, y, 30, 0, 1, b.F32, b.OS, 0) == 1     # y_pitch < out_w
-    assert b.sysconv2d_strided(x, 64, 64, 64, 0, w2, 3, 3, 2, 1, y, 31, 0, 1, b.F32, b.OS, 0) == 2     # mixed strides
+    assert b.sysconv2d_strided(x, 64, 64, 64, 0, w2, 3, 3, 2, 1, y, 31, 0, 1, b.F32, b.IS, 0) == 2     # mixed strides: output-stationary only
     assert b.sysconv2d_strided(x, 64, 64, 64, 0, w2, 3, 3, 2, 2, y, 31, 0, 1, b.F32, b.WS, 0) == 2     # WS: not built
     assert b.sysconv2d_strided(x, 64, 64, 64, 0, wi, 3, 3, 2, 2, y, 31, 0, 1, b.U8S8_S32, b.IS, 0) == 2
     w9 = np.ones((9, 9), np.float32)
-    assert b.sysconv2d_strided(x, 64, 64, 64, 0, w9, 9, 9, 2, 2, y, 28, 0, 1, b.F32, b.OS, 0) == 2     # beyond 7 x 7
+    assert b.sysconv2d_strided(x, 64, 64, 64, 0, w9, 9, 9, 2, 2, y, 28, 0, 1, b.F32, b.IS, 0) == 2     # beyond 7 x 7: output-stationary only
 
 
 def test_host_multi_argument_validation_needs_no_gpu(lib):

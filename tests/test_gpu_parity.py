@@ -720,6 +720,89 @@ def test_2d_stride2_full_hd_sampled(cuda_device):
         assert_close_f32(y.cpu().numpy()[0][rows, cols], y_ref, s_ref, "sampled, %s" % B.DESIGN_NAMES[design])
 
 
+# ------------------------------------------------------------------------ any strides (output-stationary array)
+
+
+@pytest.mark.parametrize("stride", [3, 4, 5, 7, 16, 40])
+@pytest.mark.parametrize("q", [1, 2, 3, 5, 8, 16, 31, 32])
+def test_1d_any_stride(cuda_device, stride, q):
+    for n in (q, q + 1, 777, 3 * 128 * stride + q + 5):
+        x, ws = inputs.gen_1d_f32(n, [q], seed=3300 + q + stride)
+        y = B.conv1d(torch.from_numpy(x).to(cuda_device), ws[q], B.OS, stride=stride)
+        torch.cuda.synchronize()
+        y_ref, s_ref = oracle.conv1d_f32_strided(x, ws[q], stride)
+        assert y.shape == y_ref.shape
+        assert_close_f32(y.cpu().numpy(), y_ref, s_ref, "stride %d, q=%d, n=%d" % (stride, q, n))
+
+
+def test_1d_any_stride_batch_strides_and_canaries(cuda_device):
+    q, n, batch, stride = 9, 7001, 3, 3
+    x, ws = inputs.gen_1d_f32(n * batch, [q], seed=78)
+    x = x.reshape(batch, n)
+    n_out = (n - q) // stride + 1
+    for x_off, y_off, xs, ys in [(0, 0, n, n_out), (1, 3, n + 3, n_out + 5)]:
+        xb = torch.zeros(x_off + batch * xs + 8, dtype=torch.float32, device=cuda_device)
+        yb = torch.full((y_off + batch * ys + 8,), CANARY, dtype=torch.float32, device=cuda_device)
+        xb[x_off: x_off + batch * xs].view(batch, xs)[:, :n] = torch.from_numpy(x).to(cuda_device)
+        st = B.sysconv1d_strided(xb.data_ptr() + 4 * x_off, n, xs, ws[q], q, stride, yb.data_ptr() + 4 * y_off, ys, batch,
+                                 B.F32, B.OS, torch.cuda.current_stream().cuda_stream)
+        assert st == 0, B.status_string(st)
+        torch.cuda.synchronize()
+        yh = yb.cpu().numpy()
+        body = yh[y_off: y_off + batch * ys].reshape(batch, ys)
+        assert (body[:, n_out:] == CANARY).all() and (yh[:y_off] == CANARY).all()
+        assert (yh[y_off + batch * ys:] == CANARY).all()
+        for b in range(batch):
+            y_ref, s_ref = oracle.conv1d_f32_strided(x[b], ws[q], stride)
+            assert_close_f32(body[b, :n_out], y_ref, s_ref, "signal %d" % b)
+
+
+def run_2d_strided(x_np, w_np, sr, sc, device, x_pitch=None, y_pitch=None, x_off=0, y_off=0):
+    batch, h, wd = x_np.shape
+    p, q = w_np.shape
+    oh, ow = (h - p) // sr + 1, (wd - q) // sc + 1
+    x_pitch = x_pitch or wd
+    y_pitch = y_pitch or ow
+    xb = torch.zeros(x_off + batch * h * x_pitch + 16, dtype=torch.float32, device=device)
+    yb = torch.full((y_off + batch * oh * y_pitch + 64,), CANARY, dtype=torch.float32, device=device)
+    xb[x_off: x_off + batch * h * x_pitch].view(batch, h, x_pitch)[:, :, :wd] = torch.from_numpy(x_np).to(device)
+    st = B.sysconv2d_strided(xb.data_ptr() + 4 * x_off, wd, h, x_pitch, h * x_pitch, np.ascontiguousarray(w_np), q, p,
+                             sc, sr, yb.data_ptr() + 4 * y_off, y_pitch, oh * y_pitch, batch, B.F32, B.OS,
+                             torch.cuda.current_stream().cuda_stream)
+    assert st == 0, B.status_string(st)
+    torch.cuda.synchronize()
+    yh = yb.cpu().numpy()
+    body = yh[y_off: y_off + batch * oh * y_pitch].reshape(batch, oh, y_pitch)
+    assert (body[:, :, ow:] == CANARY).all(), "write into the pitch padding"
+    assert (yh[:y_off] == CANARY).all() and (yh[y_off + batch * oh * y_pitch:] == CANARY).all()
+    for b in range(batch):
+        y_ref, s_ref = oracle.conv2d_f32_strided(x_np[b], w_np, (sr, sc))
+        assert body[b, :, :ow].shape == y_ref.shape
+        assert_close_f32(body[b, :, :ow], y_ref, s_ref, "image %d, strides (%d, %d)" % (b, sr, sc))
+
+
+@pytest.mark.parametrize("strides", [(3, 3), (2, 1), (1, 2), (2, 3), (3, 2), (4, 4), (5, 1), (1, 7), (9, 9)],
+                         ids=lambda t: "r%dc%d" % t)
+@pytest.mark.parametrize("pq", [(1, 1), (3, 3), (5, 5), (7, 7), (9, 9), (15, 15), (2, 11), (13, 4)], ids=lambda f: "%dx%d" % f)
+def test_2d_any_strides(cuda_device, strides, pq):
+    sr, sc = strides
+    x, ws = inputs.gen_2d_f32(533, 61, [pq], seed=3400 + 16 * pq[0] + pq[1] + sr, batch=2)
+    run_2d_strided(x, ws[pq], sr, sc, cuda_device)
+    run_2d_strided(x[:, :, :301], ws[pq], sr, sc, cuda_device, x_pitch=307, y_pitch=310, x_off=1, y_off=3)
+
+
+def test_2d_stride_two_large_filters_and_full_hd_stride_three(cuda_device):
+    # stride 2 beyond 7 x 7 goes to the run-time-stride array too
+    x, ws = inputs.gen_2d_f32(300, 120, [(9, 9), (15, 15), (8, 3)], seed=3500, batch=1)
+    for pq in ws:
+        run_2d_strided(x, ws[pq], 2, 2, cuda_device)
+    x, ws = inputs.gen_2d_f32(1920, 1080, [(5, 5)], seed=3501, batch=1)
+    run_2d_strided(x, ws[(5, 5)], 3, 3, cuda_device)
+    # single-output and degenerate sizes
+    x, ws = inputs.gen_2d_f32(5, 5, [(5, 5)], seed=3502, batch=3)
+    run_2d_strided(x, ws[(5, 5)], 3, 4, cuda_device)
+
+
 # ------------------------------------------------------------------------ separable 2-D convolution
 
 
