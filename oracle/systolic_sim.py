@@ -488,3 +488,128 @@ def warp_ws_1d(xs, w, lanes_per_array, R, seg_len):
         if c >= 0:
             y[:, c] = Z[last, -1]
     return y
+
+
+# ----------------------------------------------------------------------------
+# The forms the CUDA kernels actually ship beyond the plain folded passes above: the same dataflows with a
+# different choice of WHICH sums a PE-step updates together (pairs), with a whole array folded into one lane
+# (weight-stationary), and with run-time strides.  Modelled step by step so that the method, not only the
+# result, is pinned on the CPU.
+# ----------------------------------------------------------------------------
+
+
+def warp_os_1d_paired(xs, w, R):
+    """Output-stationary, PE-paired: the sums of PEs 2m and 2m+1 form a pair that ONE operation updates with
+    the same forwarded input x and the tap pair (w(t), w(t-1)): the odd PE lags one step behind the even one.
+    Q+1 steps; the first and the last touch only one sum of each pair.  Returns all 32*R sums (valid prefix
+    as for warp_os_1d)."""
+    Q = len(w)
+    assert R % 2 == 0
+    D = np.asarray(xs, dtype=np.float64).reshape(-1).copy()          # forwarded inputs, PE-major
+    n = D.size
+    Z = np.zeros(n)
+    even = np.arange(0, n, 2)
+    for t in range(Q + 1):
+        x = D[even]                                                  # the input the even PE of each pair holds
+        if t == 0:
+            Z[even] = x * w[0]
+            Z[even + 1] = 0.0
+        elif t == Q:
+            Z[even + 1] += x * w[Q - 1]
+        else:
+            Z[even] += x * w[t]
+            Z[even + 1] += x * w[t - 1]
+        if t < Q:
+            # inputs move one PE down: inside a lane by renaming, across lanes by one shuffle (lane 31 keeps its own)
+            Dn = D.copy()
+            Dn[:-1] = D[1:]
+            D = Dn
+    return Z
+
+
+def warp_is_1d_paired(xs, w, R):
+    """Input-stationary, paired: the sums of two neighbouring outputs o (even) and o+1 travel together; in PE
+    s = o + t the pair takes x(s) * (w(t), w(t-1)).  Q+1 steps.  Returns y[o] for the outputs whose whole chain
+    lies inside the tile (the first 32*R - Q of them, counted from output 0)."""
+    Q = len(w)
+    X = np.asarray(xs, dtype=np.float64).reshape(-1)
+    n = X.size
+    # pair[o/2] = (sum of output o, sum of output o+1), sitting in PE o + t after step t
+    n_pairs = (n - Q) // 2
+    first = np.zeros(n_pairs)
+    second = np.zeros(n_pairs)
+    for t in range(Q + 1):
+        for m in range(n_pairs):
+            s = 2 * m + t                                            # the PE the pair sits in at this step
+            if t == 0:
+                first[m] = X[s] * w[0]
+            elif t == Q:
+                second[m] += X[s] * w[Q - 1]
+            else:
+                first[m] += X[s] * w[t]
+                second[m] += X[s] * w[t - 1]
+    y = np.empty(2 * n_pairs)
+    y[0::2], y[1::2] = first, second
+    return y
+
+
+def warp_ws_1d_one_lane(xs, w, seg_len, n_arrays):
+    """Weight-stationary with a whole array (Q PEs) folded into ONE lane and the arrays handing their sums over
+    instead of filling and draining.  Array a streams exactly the seg_len inputs of segment a.  PE s keeps w(s);
+    at step t PE s adds x(t) * w(s) to the sum it took from PE s-1 (PE 0 opens a new sum); PE Q-1 emits.  The
+    sum of output o = t - (Q-1) of the segment is emitted at step t; for o < 0 it is the part of an output of
+    segment a-1's tail that array a's inputs contribute, and is stored there; when array a stops, the sums still
+    in flight in its PEs 1 .. Q-1 are the parts its own inputs contribute to those tail outputs, and are added.
+    The slice's last array has no successor: its tail takes the missing taps from a direct sum over the halo.
+    xs holds n_arrays*seg_len + Q - 1 inputs; returns the n_arrays*seg_len outputs."""
+    Q = len(w)
+    xs = np.asarray(xs, dtype=np.float64)
+    total = n_arrays * seg_len
+    y = np.zeros(total)
+    in_flight = np.zeros((n_arrays, Q))
+    for a in range(n_arrays):
+        Z = np.zeros(Q)
+        for t in range(seg_len):
+            x = xs[a * seg_len + t]
+            Zn = np.empty(Q)
+            Zn[0] = x * w[0]
+            Zn[1:] = Z[:-1] + x * w[1:]
+            Z = Zn
+            o = a * seg_len + t - (Q - 1)
+            if o >= 0:
+                # t >= Q-1: a complete output of this segment; t < Q-1: array a's share of a tail output of
+                # segment a-1, which array a-1 never emitted (the first array of the slice has no predecessor)
+                y[o] = Z[Q - 1]
+        in_flight[a] = Z
+    for a in range(n_arrays):
+        # PE s stopped while holding the part of output (a+1)*seg_len - 1 - s that array a's own inputs give
+        for s in range(Q - 1):
+            o = (a + 1) * seg_len - 1 - s
+            y[o] += in_flight[a][s]
+    # the last array's tail: no successor, the missing taps summed directly over the halo
+    for j in range(Q - 1):
+        o = total - 1 - j
+        for k in range(j + 1, Q):
+            y[o] += w[k] * xs[o + k]
+    return y
+
+
+def warp_os_1d_strided(xs, w, stride, n_pes):
+    """Output-stationary with any stride, residue class by residue class: for b < stride the inputs x(stride*c + b)
+    enter the PEs and move one PE down per step a, meeting the taps w(stride*a + b); the sums stay.  The last PE
+    takes its inputs from memory.  Returns the n_pes sums."""
+    Q = len(w)
+    xs = np.asarray(xs, dtype=np.float64)
+    Z = np.zeros(n_pes)
+    c = np.arange(n_pes)
+    for b in range(min(stride, Q)):
+        X = xs[stride * c + b].copy()
+        steps = (Q - b + stride - 1) // stride
+        for a in range(steps):
+            Z += X * w[stride * a + b]
+            if a + 1 < steps:
+                Xn = np.empty_like(X)
+                Xn[:-1] = X[1:]
+                Xn[-1] = xs[stride * (n_pes + a) + b]               # the array's last PE loads from memory
+                X = Xn
+    return Z

@@ -181,3 +181,59 @@ def test_warp_ws_matches_oracle(lanes, R, q, seg):
     ref, _ = oracle.conv1d_f32(xs, w)
     y = sim.warp_ws_1d(xs, w, lanes, R, seg)
     np.testing.assert_array_equal(y.reshape(-1), ref[:n_arr * seg])
+
+
+# ---- the forms the kernels ship beyond the plain folded passes: paired sums, one-lane arrays with hand-over,
+# run-time strides; integer-valued data, so every order of summation is exact
+
+
+@pytest.mark.parametrize("R", [2, 4, 20])
+@pytest.mark.parametrize("q", [1, 2, 5, 12, 13, 32])
+def test_paired_output_stationary_pass_matches_oracle(R, q):
+    rng = np.random.default_rng(100 + q)
+    xs = rng.integers(-8, 9, 32 * R).astype(np.float32)
+    w = rng.integers(-4, 5, q).astype(np.float32)
+    z = sim.warp_os_1d_paired(xs, w, R)
+    y, _ = oracle.conv1d_f32(xs, w)
+    valid = 32 * R - (q - 1)
+    np.testing.assert_array_equal(z[:valid], y[:valid])
+    np.testing.assert_array_equal(z[:valid], sim.warp_os_1d(xs, w, R)[:valid])
+
+
+@pytest.mark.parametrize("q", [1, 2, 5, 12, 13, 32])
+def test_paired_input_stationary_pass_matches_oracle(q):
+    rng = np.random.default_rng(110 + q)
+    xs = rng.integers(-8, 9, 640).astype(np.float32)
+    w = rng.integers(-4, 5, q).astype(np.float32)
+    y_pairs = sim.warp_is_1d_paired(xs, w, 20)
+    y, _ = oracle.conv1d_f32(xs, w)
+    np.testing.assert_array_equal(y_pairs, y[:y_pairs.size])
+    assert y_pairs.size >= 640 - q - 1
+
+
+@pytest.mark.parametrize("q", [1, 2, 3, 8, 31, 32])
+@pytest.mark.parametrize("seg,arrays", [(76, 32), (40, 4), (33, 2), (76, 1)])
+def test_one_lane_weight_stationary_arrays_hand_their_sums_over(q, seg, arrays):
+    if q > seg:
+        pytest.skip("array longer than a segment")
+    rng = np.random.default_rng(120 + q + seg)
+    xs = rng.integers(-8, 9, arrays * seg + q - 1).astype(np.float32)
+    w = rng.integers(-4, 5, q).astype(np.float32)
+    y = sim.warp_ws_1d_one_lane(xs, w, seg, arrays)
+    ref, _ = oracle.conv1d_f32(xs, w)
+    np.testing.assert_array_equal(y, ref)
+
+
+@pytest.mark.parametrize("stride", [1, 2, 3, 4, 7])
+@pytest.mark.parametrize("q", [1, 2, 5, 8, 32])
+def test_strided_output_stationary_array_by_residue_classes(stride, q):
+    rng = np.random.default_rng(130 + q + stride)
+    n_pes = 37
+    xs = rng.integers(-8, 9, stride * (n_pes - 1) + q + stride * 40).astype(np.float32)
+    w = rng.integers(-4, 5, q).astype(np.float32)
+    z = sim.warp_os_1d_strided(xs, w, stride, n_pes)
+    ref, _ = oracle.conv1d_f32_strided(xs, w, stride)
+    np.testing.assert_array_equal(z, ref[:n_pes])
+    if stride == 2:
+        ys, _ = sim.simulate_1d("FBS", xs[: 2 * (n_pes - 1) + q], w, stride=2)       # Table 2's own stride-2 cell
+        np.testing.assert_array_equal(z, np.asarray(ys, dtype=np.float64))
