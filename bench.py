@@ -542,6 +542,11 @@ def run_ours(args):
         scale = {"batch": args.profile_batch}
     if args.profile_filter and cfg_id in (4, 5):
         scale = dict(scale or {}, filters=[args.profile_filter])   # ncu captures only: one filter's buffers on the device
+    split = args.split_images and cfg_id == 5 and world > 1
+    if split:
+        # strong scaling: the 16 independent images are dealt out to the ranks (no collective on the data path)
+        lo, hi = shard.split_range(inputs.CONFIGS[5]["batch"], rank, world)
+        scale = dict(scale or {}, batch=max(hi - lo, 1))
     cases, keep = build_cases(cfg_id, device, scale=scale)   # every rank holds its own copy: weak scaling
     outputs_per_step = sum(c.n_out for c in cases)
 
@@ -626,14 +631,15 @@ def run_ours(args):
     line = {
         "metric": "output elements/s", "value": round(value, 3), "unit": "Gpix/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(total_ms / args.steps, 4),
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "higher_is_better": True, "scaling": "strong" if split else "weak", "vs_baseline": None,
         "dtype": "f32" if inputs.CONFIGS[cfg_id]["kind"] != "2d_u8s8" else "s32", "data": "synthetic",
         "config": {"workload": "cfg%d: %s; every filter x designs WS/OS/IS, one launch each"
                                % (cfg_id, inputs.CONFIGS[cfg_id]["note"]),
                    "launches_per_step": len(cases),
                    "l2": "flushed between steps (256 MiB write, excluded from the time)" if small
                          else "inputs larger than L2 (268 MB signal per launch)",
-                   "per_rank": "each rank convolves its own copy (independent problems, no collective)"},
+                   "per_rank": ("the 16 images are dealt out to the ranks (independent problems, no collective)" if split else
+                                "each rank convolves its own copy (independent problems, no collective)")},
         "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
     }
     if rank == 0:
@@ -885,6 +891,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle baseline leg")
+    ap.add_argument("--split-images", action="store_true",
+                    help="cfg5 on several GPUs: deal the 16 images out to the ranks (strong scaling) instead of one copy each")
     ap.add_argument("--profile-n", type=int, default=0,
                     help="ncu captures only: shrink the 1-D signal to this many samples (keep it > L2)")
     ap.add_argument("--profile-batch", type=int, default=0,

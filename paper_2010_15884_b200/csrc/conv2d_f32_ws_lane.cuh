@@ -23,6 +23,8 @@
 #pragma once
 
 #include "conv2d_f32_is_pair.cuh"
+#include "conv2d_f32_ws_reg.cuh"
+#include "conv2d_f32_ws_seg.cuh"
 
 namespace sysconv {
 
@@ -203,18 +205,26 @@ cudaError_t launch_conv2d_ws_lane(const Conv2DArgs &a, const Taps2D &taps, cudaS
     return cudaGetLastError();
 }
 
-// fp32 runs the one-lane-per-array paired kernel; the four-lane arrays of conv2d_ws_kernel serve the integer
-// data and the images too small to give the one-warp CTAs of the paired kernel a few warps per SM
-// (1920 x 1080, 5 x 5: 25 us against 36 us)
+// fp32 dispatch.  Small filters (at most 8 columns, P*Q up to about 32): the all-register form with the arrays side by
+// side along the rows (conv2d_f32_ws_reg.cuh).  Larger filters: the arrays stacked over the rows with transposed
+// staging (this file) when the problem gives its one-warp blocks a few warps per SM, else the segment form with
+// the hand-over in shared memory (conv2d_f32_ws_seg.cuh), which reads its inputs straight from memory and so suits
+// problems that live in L2 (1920 x 1080, 5 x 5: 13 us against 20 us for four-lane arrays with register taps).
+// None of the three pads with zero taps: an input outside an output's window never enters its sum.
 template <int P, int Q>
 struct FastPath2D<F32Traits, SYSCONV_WS, P, Q> {
     static bool launch(const Conv2DArgs &a, const Taps2D &taps, cudaStream_t s, cudaError_t *err)
     {
-        const long long bands = (a.out_h + kWlRows - 1) / kWlRows;
-        const long long max_segs = (a.out_w + 127) / 128;
-        if (bands * max_segs * a.batch < 148LL * 4) return false;
-        *err = launch_conv2d_ws_lane<P, Q>(a, taps, s);
-        return true;
+        if constexpr (WsrShape<P, Q>::kFits) {
+            *err = launch_conv2d_ws_reg<P, Q>(a, taps, s);
+            return true;
+        } else {
+            const long long bands = (a.out_h + kWlRows - 1) / kWlRows;
+            const long long max_segs = (a.out_w + 127) / 128;
+            if (bands * max_segs * a.batch < 148LL * 4) *err = launch_conv2d_ws_seg<P, Q>(a, taps, s);
+            else *err = launch_conv2d_ws_lane<P, Q>(a, taps, s);
+            return true;
+        }
     }
 };
 

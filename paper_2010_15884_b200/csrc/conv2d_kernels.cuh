@@ -730,7 +730,8 @@ cudaError_t launch_conv2d_pq(const Conv2DArgs &a, const typename Tr::taps_t &tap
         cudaError_t err = cudaSuccess;
         if (FastPath2D<Tr, DESIGN, P, Q>::launch(a, taps, s, &err)) return err;
     }
-    if (DESIGN == SYSCONV_WS) {
+    if constexpr (DESIGN == SYSCONV_WS && !std::is_same<Tr, F32Traits>::value) {
+        // (integer data; fp32 has its own weight-stationary kernels behind the hook above)
         // CTAs = width segments x bands of 128 rows x images; segments are multiples of 32 columns and as
         // long as possible (each costs QP-1 fill steps) while still giving a few CTAs per SM
         const long long bands = (a.out_h + kWsRows2 - 1) / kWsRows2;
@@ -746,6 +747,7 @@ cudaError_t launch_conv2d_pq(const Conv2DArgs &a, const typename Tr::taps_t &tap
         launch_kernel(conv2d_ws_kernel<Tr, P, Q>, grid, kThreads2, s, a, taps, seg_w);
         return cudaGetLastError();
     }
+    if constexpr (DESIGN == SYSCONV_WS) return kNoInstantiation;
     using Sh = Shape2D<Tr, DESIGN, P, Q>;
     if constexpr (std::is_same<Tr, F32Traits>::value && DESIGN == SYSCONV_OS && P >= 6)
         return launch_conv2d_os_rowpair<P, Q>(a, taps.w, s);
