@@ -376,8 +376,10 @@ struct IsGeom {
 // The P-deep input column of a PE is a window that slides down one row per output row.  Where the code stays
 // small the row loop is unrolled P times and the window is a ring (input row r+p sits in slot (u+p) mod P, u =
 // position in the unrolled group), so sliding costs nothing; otherwise the window is shifted by (P-1)*R moves.
+// (Measured: the ring pays for the four-PE-per-lane kernels of the small problems -- 1920 x 1080, 5 x 5: 7.9 -> 6.4 us;
+// with eight PEs per lane its registers cost residency -- 16 x 4096^2, 3 x 3: 0.39 -> 0.45 ms -- so those shift.)
 template <int P, int Q, int R>
-constexpr bool kIsRing = P > 1 && P * P * Q * R <= 2048;
+constexpr bool kIsRing = P > 1 && R == 4 && P * P * Q * R <= 2048;
 
 template <typename Tr, int P, int Q, int R, int MIN_CTAS>
 __global__ void __launch_bounds__(kThreads2, MIN_CTAS)
