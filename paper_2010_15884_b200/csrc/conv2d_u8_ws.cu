@@ -1,6 +1,6 @@
 // 2-D uint8 x int8 -> int32 kernels of the weight-stationary (derived from BSM) design, filter heights 1..10 (all widths 1..15); the taller
 // filters are compiled in conv2d_u8_ws_hi.cu so that the two halves build in parallel.
-#include "conv2d_kernels.cuh"
+#include "conv2d_u8_ws_dp4a.cuh"
 
 namespace sysconv {
 

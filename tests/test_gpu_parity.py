@@ -466,9 +466,9 @@ def test_2d_f32_small_problems(cuda_device, design, pq, size):
     assert B.device_status() == 0
 
 
-@pytest.mark.parametrize("design", [B.OS, B.IS], ids=_ids)
-@pytest.mark.parametrize("pq", [(3, 3), (7, 7), (1, 1), (5, 13), (7, 15), (2, 4)], ids=lambda f: "%dx%d" % f)
-@pytest.mark.parametrize("size", [(1101, 83, 2), (3840, 140, 1), (1000, 41, 1), (4097, 64, 1), (64, 20, 3)],
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+@pytest.mark.parametrize("pq", [(3, 3), (7, 7), (1, 1), (5, 13), (7, 15), (2, 4), (15, 15), (11, 9)], ids=lambda f: "%dx%d" % f)
+@pytest.mark.parametrize("size", [(1101, 83, 2), (3840, 140, 1), (1000, 41, 1), (4097, 64, 1), (64, 20, 3), (496, 35, 1), (497, 36, 2)],
                          ids=lambda t: "%dx%dx%d" % t)
 def test_2d_u8_small_problems(cuda_device, design, pq, size):
     wd, h, batch = size
@@ -1182,13 +1182,13 @@ def test_2d_u8_shapes_and_extremes(cuda_device, design, pq):
         check_2d(xm, np.full(pq, v, np.int8), design, cuda_device)
 
 
-@pytest.mark.parametrize("design", [B.OS, B.IS], ids=_ids)
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
 @pytest.mark.parametrize("pq", [(1, 1), (3, 3), (5, 5), (7, 7), (7, 15), (8, 15), (15, 15), (9, 2), (4, 13), (12, 8),
                                 (1, 4), (2, 5), (6, 9), (7, 12), (3, 8)], ids=lambda f: "%dx%d" % f)
 def test_2d_u8_packed_rows(cuda_device, design, pq):
     """Rows that start 4-byte aligned take the packed four-taps-per-step kernels (OS: every filter size; IS: up to
-    seven filter rows): several strips, a ragged right edge, pitch padding, unaligned outputs, and the extreme
-    pixel/tap values."""
+    seven filter rows; WS: rows aligned to 16 bytes): several strips, a ragged right edge, pitch padding, unaligned
+    outputs, and the extreme pixel/tap values."""
     p, q = pq
     x, ws = inputs.gen_2d_u8s8(1101, 41, [pq], seed=90 + p + q, batch=2)
     check_2d(x, ws[pq], design, cuda_device, x_pitch=1104)
