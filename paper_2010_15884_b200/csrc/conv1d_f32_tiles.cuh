@@ -19,9 +19,12 @@
 // last PE takes its input from memory) cut every chain at the array's edge.
 //
 // Every lane serves U arrays (the same PE of U different signals) per pass, so that U independent chains overlap
-// in the pipelines and U times as many bytes are in flight.  The signals of a pass are staged in shared memory by
-// the lanes of their own arrays ("memory" of the recurrences = this staging area), the outputs go back the same
-// way, and the global accesses of a warp cover one contiguous run of signals.
+// in the pipelines.  The signals of a pass are staged in shared memory ("memory" of the recurrences = this staging
+// area) and the outputs go back the same way.  Densely packed signals (the usual case: signal g starts right after
+// signal g-1, 16-byte aligned) make one contiguous run per pass, which moves as whole 128-bit words, and the
+// words of the NEXT pass are fetched into registers before the current pass is computed, so that the memory
+// latency is overlapped with the arithmetic of the same warp.  Any other layout is gathered signal by signal by
+// the lanes of each array.
 #pragma once
 
 #include "sysconv_common.cuh"
@@ -32,6 +35,7 @@ constexpr int kTilesMaxQ = 8;           // filter lengths 1 .. 8
 constexpr int kTilesMaxOut = 32;        // outputs per signal 1 .. 32
 constexpr int kTilesWarps = 4;
 constexpr int kTilesFloatsPerWarp = 2560;   // staging area of one warp (inputs + outputs of a pass)
+constexpr int kTilesVecPerLane = 6;         // dense form: 128-bit words of a pass's inputs per lane (at most 768 floats per pass)
 
 // PEs of one array of a design for C outputs and Q taps
 inline int tiles_array_pes(int design, int c, int q)
@@ -44,9 +48,9 @@ inline int tiles_array_pes(int design, int c, int q)
     }
 }
 
-template <int DESIGN, int Q, int U>
+template <int DESIGN, int Q, int U, bool DENSE>
 __global__ void __launch_bounds__(kTilesWarps *kLanes)
-conv1d_tiles_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, const int LA, const int AW)
+conv1d_tiles_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, const int LA, const int AW, const int warp_floats)
 {
     dependent_launch_enter();
     extern __shared__ __align__(16) float tiles_smem[];
@@ -56,16 +60,34 @@ conv1d_tiles_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, con
     const int arr = lane / LA;                  // array this lane belongs to (>= AW: the lane idles)
     const int pe = lane - arr * LA;             // its PE in that array
     const bool member = arr < AW;
-    float *s_in = tiles_smem + warp * (U * AW * (N + C));
+    float *s_in = tiles_smem + warp * warp_floats;
     float *s_out = s_in + U * AW * N;
     const float *xg = static_cast<const float *>(a.x);
     float *yg = static_cast<float *>(a.y);
     const long long per_pass = static_cast<long long>(U) * AW;              // signals one warp takes per pass
     const long long stride = static_cast<long long>(gridDim.x) * kTilesWarps * per_pass;
+    const int in_vec = U * AW * N / 4, out_vec = U * AW * C / 4;            // dense form: 128-bit words per pass
 
-    for (long long g0 = (static_cast<long long>(blockIdx.x) * kTilesWarps + warp) * per_pass; g0 < a.batch; g0 += stride) {
-        // ---- the signals of this pass enter the staging area, each fetched by the lanes of its own array
-        if (member) {
+    // dense form: the inputs of a whole pass are one contiguous, 16-byte aligned run
+    float4 pre[kTilesVecPerLane];
+    auto fetch = [&](long long g) {
+        const float4 *src = reinterpret_cast<const float4 *>(xg + g * N);
+#pragma unroll
+        for (int i = 0; i < kTilesVecPerLane; ++i)
+            if (lane + kLanes * i < in_vec) pre[i] = __ldg(src + lane + kLanes * i);
+    };
+    long long g0 = (static_cast<long long>(blockIdx.x) * kTilesWarps + warp) * per_pass;
+    bool have = DENSE && g0 + per_pass <= a.batch;      // a whole pass: its words are in flight or in registers
+    if (have) fetch(g0);
+
+    for (; g0 < a.batch; g0 += stride) {
+        // ---- the signals of this pass enter the staging area
+        if (DENSE && have) {
+#pragma unroll
+            for (int i = 0; i < kTilesVecPerLane; ++i)
+                if (lane + kLanes * i < in_vec) reinterpret_cast<float4 *>(s_in)[lane + kLanes * i] = pre[i];
+        } else if (member) {
+            // each signal fetched by the lanes of its own array
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const long long g = g0 + u * AW + arr;
@@ -73,41 +95,42 @@ conv1d_tiles_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, con
                     for (int k = pe; k < N; k += LA) s_in[(u * AW + arr) * N + k] = __ldg(xg + g * a.x_bstride + k);
             }
         }
-        __syncwarp();
-        const float *xin[U];
-        float *yout[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int slot = u * AW + (member ? arr : 0);
-            xin[u] = s_in + slot * N;
-            yout[u] = s_out + slot * C;
+        bool have_next = false;
+        if (DENSE) {
+            have_next = g0 + stride + per_pass <= a.batch;
+            if (have_next) fetch(g0 + stride);          // in flight while this pass is computed
         }
+        __syncwarp();
+        // signal u of this lane's array: inputs xin0[u * xu + k], outputs yout0[u * yu + k]
+        const float *xin0 = s_in + (member ? arr : 0) * N;
+        float *yout0 = s_out + (member ? arr : 0) * C;
+        const int xu = AW * N, yu = AW * C;
 
         if (DESIGN == SYSCONV_OS) {
             // FBS: PE c keeps Z(c); inputs move one PE down per step, the last PE takes x(c+q) from memory
             float X[U], Z[U];
 #pragma unroll
-            for (int u = 0; u < U; ++u) X[u] = pe < C ? xin[u][pe] : 0.f;
+            for (int u = 0; u < U; ++u) X[u] = pe < C ? xin0[u * xu + pe] : 0.f;
 #pragma unroll
             for (int t = 0; t < Q; ++t) {
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
                     if (t > 0) {
                         const float fwd = __shfl_down_sync(kFullMask, X[u], 1);
-                        X[u] = (pe == C - 1) ? xin[u][pe + t] : fwd;
+                        X[u] = (pe == C - 1) ? xin0[u * xu + pe + t] : fwd;
                     }
                     Z[u] = t == 0 ? X[u] * taps.w[0] : fmaf(X[u], taps.w[t], Z[u]);
                 }
             }
             if (member && pe < C) {
 #pragma unroll
-                for (int u = 0; u < U; ++u) yout[u][pe] = Z[u];
+                for (int u = 0; u < U; ++u) yout0[u * yu + pe] = Z[u];
             }
         } else if (DESIGN == SYSCONV_IS) {
             // SBM: PE s keeps x(s); the sums move one PE up per step; PE s >= Q-1 ends with y(s-(Q-1))
             float X[U], Z[U];
 #pragma unroll
-            for (int u = 0; u < U; ++u) X[u] = pe < N ? xin[u][pe] : 0.f;
+            for (int u = 0; u < U; ++u) X[u] = pe < N ? xin0[u * xu + pe] : 0.f;
 #pragma unroll
             for (int t = 0; t < Q; ++t) {
 #pragma unroll
@@ -122,7 +145,7 @@ conv1d_tiles_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, con
             }
             if (member && pe >= Q - 1 && pe < N) {
 #pragma unroll
-                for (int u = 0; u < U; ++u) yout[u][pe - (Q - 1)] = Z[u];
+                for (int u = 0; u < U; ++u) yout0[u * yu + pe - (Q - 1)] = Z[u];
             }
         } else if (DESIGN == SYSCONV_WS) {
             // BSM: PE s keeps w(s); x(t) is broadcast to the array; the sums move one PE up; the last PE emits
@@ -134,8 +157,8 @@ conv1d_tiles_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, con
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
                     const float up = __shfl_up_sync(kFullMask, Z[u], 1);
-                    Z[u] = fmaf(xin[u][t], w, pe == 0 ? 0.f : up);
-                    if (member && pe == Q - 1 && t >= Q - 1) yout[u][t - (Q - 1)] = Z[u];
+                    Z[u] = fmaf(xin0[u * xu + t], w, pe == 0 ? 0.f : up);
+                    if (member && pe == Q - 1 && t >= Q - 1) yout0[u * yu + t - (Q - 1)] = Z[u];
                 }
             }
         } else if (DESIGN == SYSCONV_FSM) {
@@ -153,9 +176,9 @@ conv1d_tiles_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, con
                     const float z_fwd = __shfl_down_sync(kFullMask, Z[u], 1);
                     Xprev[u] = X[u];
                     if (active) {
-                        X[u] = (c == 0 || pe == Q - 1) ? xin[u][c + pe] : x_fwd;
+                        X[u] = (c == 0 || pe == Q - 1) ? xin0[u * xu + c + pe] : x_fwd;
                         Z[u] = (pe == Q - 1) ? X[u] * w : fmaf(X[u], w, z_fwd);
-                        if (member && pe == 0) yout[u][c] = Z[u];
+                        if (member && pe == 0) yout0[u * yu + c] = Z[u];
                     }
                 }
             }
@@ -172,12 +195,12 @@ conv1d_tiles_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, con
                 for (int u = 0; u < U; ++u) {
                     const float fwd = __shfl_up_sync(kFullMask, W[u], 1);
                     W[u] = pe == 0 ? w_in : fwd;
-                    if (active) Z[u] = q == 0 ? xin[u][t] * W[u] : fmaf(xin[u][t], W[u], Z[u]);
+                    if (active) Z[u] = q == 0 ? xin0[u * xu + t] * W[u] : fmaf(xin0[u * xu + t], W[u], Z[u]);
                 }
             }
             if (member && pe < C) {
 #pragma unroll
-                for (int u = 0; u < U; ++u) yout[u][pe] = Z[u];
+                for (int u = 0; u < U; ++u) yout0[u * yu + pe] = Z[u];
             }
         } else {
             // FFS: PE c keeps Z(c); inputs move one PE up per step, weights one PE up every two steps; t = 2c + q
@@ -194,7 +217,7 @@ conv1d_tiles_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, con
                     const float w_fwd = __shfl_up_sync(kFullMask, Wprev[u], 1);
                     Wprev[u] = W[u];
                     if (active) {
-                        X[u] = (pe == 0 || q == Q - 1) ? xin[u][pe + q] : x_fwd;
+                        X[u] = (pe == 0 || q == Q - 1) ? xin0[u * xu + pe + q] : x_fwd;
                         W[u] = pe == 0 ? w_in : w_fwd;
                         Z[u] = q == 0 ? X[u] * W[u] : fmaf(X[u], W[u], Z[u]);
                     }
@@ -202,12 +225,17 @@ conv1d_tiles_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, con
             }
             if (member && pe < C) {
 #pragma unroll
-                for (int u = 0; u < U; ++u) yout[u][pe] = Z[u];
+                for (int u = 0; u < U; ++u) yout0[u * yu + pe] = Z[u];
             }
         }
         __syncwarp();
         // ---- the outputs of this pass leave the staging area the way the inputs came
-        if (member) {
+        if (DENSE && have) {
+            float4 *dst = reinterpret_cast<float4 *>(yg + g0 * C);
+#pragma unroll
+            for (int i = 0; i < kTilesVecPerLane; ++i)
+                if (lane + kLanes * i < out_vec) dst[lane + kLanes * i] = reinterpret_cast<const float4 *>(s_out)[lane + kLanes * i];
+        } else if (member) {
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const long long g = g0 + u * AW + arr;
@@ -215,6 +243,8 @@ conv1d_tiles_kernel(const Conv1DArgs a, const __grid_constant__ Taps1D taps, con
                     for (int k = pe; k < C; k += LA) yg[g * a.y_bstride + k] = s_out[(u * AW + arr) * C + k];
             }
         }
+        have = have_next;
+        // (the next pass refills the staging area only after the barrier that follows its own input stores)
         __syncwarp();
     }
 }
@@ -226,15 +256,12 @@ inline bool tiles_eligible(const Conv1DArgs &a, int design, int q)
     return tiles_array_pes(design, static_cast<int>(a.n_out), q) <= kLanes;
 }
 
-template <int DESIGN, int Q>
-cudaError_t launch_conv1d_tiles_q(const Conv1DArgs &a, const Taps1D &taps, cudaStream_t s)
+template <int DESIGN, int Q, int U>
+cudaError_t launch_conv1d_tiles_u(const Conv1DArgs &a, const Taps1D &taps, int LA, int AW, bool dense, cudaStream_t s)
 {
     const int C = static_cast<int>(a.n_out), N = static_cast<int>(a.n);
-    const int LA = tiles_array_pes(DESIGN, C, Q);
-    const int AW = kLanes / LA;
-    const int per_slot = AW * (N + C);
-    const int U = per_slot * 4 <= kTilesFloatsPerWarp ? 4 : per_slot * 2 <= kTilesFloatsPerWarp ? 2 : 1;
-    const size_t smem = sizeof(float) * kTilesWarps * U * per_slot;
+    const int warp_floats = (U * AW * (N + C) + 3) / 4 * 4;
+    const size_t smem = sizeof(float) * kTilesWarps * warp_floats;
     const long long per_block = static_cast<long long>(kTilesWarps) * U * AW;
     long long blocks = (a.batch + per_block - 1) / per_block;
     if (blocks > 148LL * 16) blocks = 148LL * 16;           // the warps loop over the remaining signals
@@ -248,10 +275,31 @@ cudaError_t launch_conv1d_tiles_q(const Conv1DArgs &a, const Taps1D &taps, cudaS
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = dependent_launch_enabled() ? 1 : 0;
-    if (U == 4) cudaLaunchKernelEx(&cfg, conv1d_tiles_kernel<DESIGN, Q, 4>, a, taps, LA, AW);
-    else if (U == 2) cudaLaunchKernelEx(&cfg, conv1d_tiles_kernel<DESIGN, Q, 2>, a, taps, LA, AW);
-    else cudaLaunchKernelEx(&cfg, conv1d_tiles_kernel<DESIGN, Q, 1>, a, taps, LA, AW);
+    if (dense) cudaLaunchKernelEx(&cfg, conv1d_tiles_kernel<DESIGN, Q, U, true>, a, taps, LA, AW, warp_floats);
+    else cudaLaunchKernelEx(&cfg, conv1d_tiles_kernel<DESIGN, Q, U, false>, a, taps, LA, AW, warp_floats);
     return cudaGetLastError();
+}
+
+template <int DESIGN, int Q>
+cudaError_t launch_conv1d_tiles_q(const Conv1DArgs &a, const Taps1D &taps, cudaStream_t s)
+{
+    const int C = static_cast<int>(a.n_out), N = static_cast<int>(a.n);
+    const int LA = tiles_array_pes(DESIGN, C, Q);
+    const int AW = kLanes / LA;
+    // signals per lane and pass: as many as the staging area and the registers of the dense form take
+    int U = 16;
+    while (U > 1 && (U * AW * (N + C) > kTilesFloatsPerWarp || U * AW * N > kTilesVecPerLane * kLanes * 4)) U /= 2;
+    // dense form: signals packed back to back, every pass a 16-byte aligned run of whole 128-bit words
+    const unsigned long long xa = reinterpret_cast<unsigned long long>(a.x), ya = reinterpret_cast<unsigned long long>(a.y);
+    const bool dense = a.x_bstride == N && a.y_bstride == C && (xa & 15ull) == 0 && (ya & 15ull) == 0 &&
+                       (U * AW * N) % 4 == 0 && (U * AW * C) % 4 == 0 && U * AW * N <= kTilesVecPerLane * kLanes * 4;
+    switch (U) {
+        case 16: return launch_conv1d_tiles_u<DESIGN, Q, 16>(a, taps, LA, AW, dense, s);
+        case 8: return launch_conv1d_tiles_u<DESIGN, Q, 8>(a, taps, LA, AW, dense, s);
+        case 4: return launch_conv1d_tiles_u<DESIGN, Q, 4>(a, taps, LA, AW, dense, s);
+        case 2: return launch_conv1d_tiles_u<DESIGN, Q, 2>(a, taps, LA, AW, dense, s);
+        default: return launch_conv1d_tiles_u<DESIGN, Q, 1>(a, taps, LA, AW, dense, s);
+    }
 }
 
 template <int DESIGN>

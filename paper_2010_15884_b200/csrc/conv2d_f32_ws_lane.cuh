@@ -36,6 +36,8 @@ constexpr int kWlRows = kLanes * kWlM;          // 128 output rows per CTA (one 
 template <int P, int Q>
 struct WlShape {
     static constexpr int kChunk = P * Q <= 25 ? 16 : 8;
+    // how the multiply-adds of a macro-step are written out (see the kernel): 1 = sub-step outermost, 0 = chain by chain
+    static constexpr int kOrder = P >= 12 ? 1 : 0;
 };
 constexpr int kWlPitch = 164;                   // rows per staged column: >= 128 + 14, = 4 mod 32 (conflict-free transposes)
 constexpr int kWlPitchO = 132;                  // rows per column of the output ring: >= 128, = 4 mod 32
@@ -154,17 +156,43 @@ conv2d_ws_lane_kernel(const Conv2DArgs a, const __grid_constant__ Taps2D taps, c
                     *reinterpret_cast<float4 *>(s_o + ((o + 1) & (kWlRing - 1)) * kWlPitchO + 4 * lane) =
                         make_float4(e1[0], e1[1], e1[2], e1[3]);
                 }
+                // The pairs move one PE up (register renaming), then the P sub-steps of macro-step T in every PE.  The
+                // order in which the independent chains (rows x PEs) are written matters to the compiler's schedule.
+                // Tall filters: sub-step outermost, the tap pair of (p, s) serves the four rows and all chains
+                // advance side by side (15x15: 74 against 61 % of the FP32 peak); smaller ones: chain by chain (9x9: 64 against
+                // 52 % the other way round).
+#pragma unroll
+                for (int m = 0; m < M; ++m)
+#pragma unroll
+                    for (int s = Q - 1; s >= 1; --s)
+                        if (s % 2 == v) Z[m][s] = Z[m][s - 1];
+                if constexpr (WlShape<P, Q>::kOrder == 1) {
+#pragma unroll
+                    for (int p = 0; p < P; ++p) {
+#pragma unroll
+                        for (int s = Q - 1; s >= 1; --s) {
+                            if (s % 2 != v) continue;
+                            const float2 w2 = tp.w[p * (Q + 1) + s];
+#pragma unroll
+                            for (int m = 0; m < M; ++m)
+                                Z[m][s] = __ffma2_rn(make_float2(xk[m + p], xk[m + p]), w2, Z[m][s]);
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int m = 0; m < M; ++m)
+#pragma unroll
+                        for (int s = Q - 1; s >= 1; --s) {
+                            if (s % 2 != v) continue;
+                            float2 z = Z[m][s];
+#pragma unroll
+                            for (int p = 0; p < P; ++p)
+                                z = __ffma2_rn(make_float2(xk[m + p], xk[m + p]), tp.w[p * (Q + 1) + s], z);
+                            Z[m][s] = z;
+                        }
+                }
 #pragma unroll
                 for (int m = 0; m < M; ++m) {
-#pragma unroll
-                    for (int s = Q - 1; s >= 1; --s) {
-                        if (s % 2 != v) continue;
-                        float2 z = Z[m][s - 1];
-#pragma unroll
-                        for (int p = 0; p < P; ++p)     // sub-steps p of macro-step T
-                            z = __ffma2_rn(make_float2(xk[m + p], xk[m + p]), tp.w[p * (Q + 1) + s], z);
-                        Z[m][s] = z;
-                    }
                     if (v == 0) {
                         float z = xk[m] * taps.w[0];    // PE 0 opens a pair: filter column 0, first sum only
 #pragma unroll

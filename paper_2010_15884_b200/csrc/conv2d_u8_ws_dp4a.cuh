@@ -26,6 +26,7 @@ constexpr int kU8WsWarps = 4;
 constexpr int kU8WsSeg = 16;                    // pixels per array and pass (one 128-bit load)
 constexpr int kU8WsOut = (kLanes - 1) * kU8WsSeg;
 constexpr int kU8WsPitch = kU8WsSeg + 4;        // ints per lane block of the output staging row
+constexpr int kU8WsUnrollP = 7;                 // filters up to this height: every input row of a pass unrolled
 
 template <int P, int Q>
 __global__ void __launch_bounds__(kU8WsWarps *kLanes)
@@ -56,8 +57,10 @@ conv2d_u8_ws_dp4a_kernel(const Conv2DArgs a, const __grid_constant__ TapsPacked 
         for (int m = 0; m < M; ++m)
 #pragma unroll
             for (int c = 0; c < SEG + TAIL; ++c) acc[m][c] = 0;
-#pragma unroll
-        for (int kk = 0; kk < K; ++kk) {
+        // One input row: fetched once, its 16 shifted words built once, used by every output row it reaches.  FULL:
+        // the row reaches all four output rows (kk in [M-1, P-1]), through the filter rows kk-m.
+        auto input_row = [&](auto full_tag, int kk) {
+            constexpr bool FULL = decltype(full_tag)::value;
             const uint8_t *rowp = xb + static_cast<long long>(min(rg + kk, a.height - 1)) * a.x_pitch + col0;
             unsigned W[5];
             if (whole) {
@@ -74,6 +77,11 @@ conv2d_u8_ws_dp4a_kernel(const Conv2DArgs a, const __grid_constant__ TapsPacked 
                 }
             }
             W[4] = __shfl_down_sync(kFullMask, W[0], 1);        // the first pixels of the next segment
+            int wt[M][G];                                       // the taps through which this row reaches the four output rows
+#pragma unroll
+            for (int m = 0; m < M; ++m)
+#pragma unroll
+                for (int g = 0; g < G; ++g) wt[m][g] = (FULL || (kk - m >= 0 && kk - m < P)) ? taps.w[(kk - m) * 4 + g] : 0;
 #pragma unroll
             for (int t = 0; t < SEG; ++t) {
                 // the broadcast input of macro-step t: the four pixels starting at pixel t of the segment
@@ -81,13 +89,24 @@ conv2d_u8_ws_dp4a_kernel(const Conv2DArgs a, const __grid_constant__ TapsPacked 
                 const unsigned xw = sh == 0 ? W[j] : __byte_perm(W[j], W[j + 1], sh == 1 ? 0x4321 : sh == 2 ? 0x5432 : 0x6543);
 #pragma unroll
                 for (int m = 0; m < M; ++m) {
-                    const int p = kk - m;                       // the filter row through which input row rg+kk reaches output row rg+m
-                    if (p < 0 || p >= P) continue;
+                    if (!FULL && (kk - m < 0 || kk - m >= P)) continue;     // (kk is a constant where FULL is false)
 #pragma unroll
                     for (int g = 0; g < G; ++g)                 // word-PE g works on output column t - 4g
-                        acc[m][TAIL + t - 4 * g] = dp4a_u8s8(xw, taps.w[p * 4 + g], acc[m][TAIL + t - 4 * g]);
+                        acc[m][TAIL + t - 4 * g] = dp4a_u8s8(xw, wt[m][g], acc[m][TAIL + t - 4 * g]);
                 }
             }
+        };
+        if constexpr (P <= kU8WsUnrollP) {
+#pragma unroll
+            for (int kk = 0; kk < K; ++kk) input_row(std::false_type{}, kk);
+        } else {
+            // tall filters: the rows that reach all four output rows run in a loop (code size), the others unrolled
+#pragma unroll
+            for (int kk = 0; kk < M - 1; ++kk) input_row(std::false_type{}, kk);
+#pragma unroll 1
+            for (int kk = M - 1; kk < P; ++kk) input_row(std::true_type{}, kk);
+#pragma unroll
+            for (int kk = P; kk < K; ++kk) input_row(std::false_type{}, kk);
         }
         // the successor's share of this segment's last TAIL outputs comes back by shuffle
 #pragma unroll
