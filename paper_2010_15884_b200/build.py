@@ -1,7 +1,8 @@
 """Build libsysconv.so in-tree with nvcc for sm_100a.
 
 ``python -m paper_2010_15884_b200.build`` compiles every ``csrc/*.cu`` to an
-object (in parallel, only when the source or a header is newer than the object)
+object (in parallel, only when the source or one of the headers it includes,
+as recorded by the compiler in a dependency file, is newer than the object)
 and links them into ``paper_2010_15884_b200/libsysconv.so``.  No GPU is needed.
 """
 import concurrent.futures
@@ -35,9 +36,34 @@ def _newest_header():
     return max(os.path.getmtime(p) for p in deps)
 
 
+def _recorded_deps(obj):
+    """Files the object was compiled from, read from the dependency file nvcc wrote beside it (None if absent)."""
+    dep = obj + ".d"
+    if not os.path.exists(dep):
+        return None
+    with open(dep) as f:
+        words = f.read().replace("\\\n", " ").split()
+    files = [os.path.normpath(os.path.join(CSRC, w)) for w in words[1:] if not w.endswith(":")]
+    root = os.path.abspath(os.path.join(HERE, ".."))
+    mine = [w for w in files if w.startswith(root)]     # this repository's sources and headers; not the toolkit's
+    return mine or None
+
+
+def _stale(src, obj, hdr_time):
+    if not os.path.exists(obj):
+        return True
+    built = os.path.getmtime(obj)
+    if built < max(os.path.getmtime(src), os.path.getmtime(os.path.abspath(__file__))):
+        return True
+    deps = _recorded_deps(obj)
+    if deps is None:
+        return built < hdr_time             # no record: any newer header counts
+    return any((not os.path.exists(d)) or os.path.getmtime(d) > built for d in deps)
+
+
 def _compile(src, obj, verbose):
-    cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]
-    res = subprocess.run(cmd, capture_output=True, text=True)
+    cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-MD", "-MF", obj + ".d", "-c", src, "-o", obj]
+    res = subprocess.run(cmd, capture_output=True, text=True, cwd=CSRC)
     if res.returncode != 0:
         raise RuntimeError("nvcc failed for %s:\n%s\n%s" % (src, res.stdout, res.stderr))
     return res.stderr
@@ -54,7 +80,7 @@ def build(force=False, verbose=False, jobs=None):
     for src in sources:
         obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
         objs.append(obj)
-        if force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), hdr_time):
+        if force or _stale(src, obj, hdr_time):
             todo.append((src, obj))
     if todo:
         jobs = jobs or min(len(todo), os.cpu_count() or 4)

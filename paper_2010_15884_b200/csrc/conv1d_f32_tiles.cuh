@@ -286,8 +286,10 @@ cudaError_t launch_conv1d_tiles_q(const Conv1DArgs &a, const Taps1D &taps, cudaS
     const int C = static_cast<int>(a.n_out), N = static_cast<int>(a.n);
     const int LA = tiles_array_pes(DESIGN, C, Q);
     const int AW = kLanes / LA;
-    // signals per lane and pass: as many as the staging area and the registers of the dense form take
-    int U = 16;
+    // signals per lane and pass: as many as the staging area and the registers of the dense form take for the two
+    // short-schedule designs (FBS filter 5, 10.5 M signals: 310 / 416 / 483 / 531 Gpix/s with 2 / 4 / 8 / 16); the
+    // designs that idle through CheckTime steps run best with two (BFS: 76 against 42 with 16, FFS: 34 against 15)
+    int U = (DESIGN == SYSCONV_OS || DESIGN == SYSCONV_IS || DESIGN == SYSCONV_WS) ? 16 : 2;
     while (U > 1 && (U * AW * (N + C) > kTilesFloatsPerWarp || U * AW * N > kTilesVecPerLane * kLanes * 4)) U /= 2;
     // dense form: signals packed back to back, every pass a 16-byte aligned run of whole 128-bit words
     const unsigned long long xa = reinterpret_cast<unsigned long long>(a.x), ya = reinterpret_cast<unsigned long long>(a.y);
