@@ -899,7 +899,17 @@ def main():
                     help="ncu captures only: shrink configuration 5 to this many images")
     ap.add_argument("--profile-filter", type=int, default=0,
                     help="ncu captures only: keep one filter size of configuration 4 or 5 (only its buffers are allocated)")
+    ap.add_argument("--paper-experiment", action="store_true",
+                    help="only the table of the paper's own experiment (10.5 M signals of 16 outputs, six designs); "
+                         "also the command the ncu capture of the tiny-signal kernel runs")
     args = ap.parse_args()
+    if args.paper_experiment:
+        import torch
+        from paper_2010_15884_b200 import binding as B
+        B.load_library()
+        rows = six_designs_table(torch.device("cuda", 0), args.detail_reps, measured_peaks()[0])
+        print(json.dumps({"six_designs_paper_experiment": rows}))
+        return
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if args.impl == "reference":
