@@ -59,20 +59,19 @@ def run_1d(x_np, w_np, design, device, batch_stride=None, offset=0):
     n_out = n - q + 1
     xs = batch_stride or n
     ys = (batch_stride or n_out)
-    xbuf = torch.zeros(offset + batch * xs + 8, dtype=torch.float32, device=device)
+    xh = np.zeros(offset + batch * xs + 8, dtype=np.float32)
+    np.lib.stride_tricks.as_strided(xh[offset:], shape=(batch, n), strides=(4 * xs, 4))[...] = x2
+    xbuf = torch.from_numpy(xh).to(device)
     ybuf = torch.full((offset + batch * ys + 64,), CANARY, dtype=torch.float32, device=device)
-    for b in range(batch):
-        xbuf[offset + b * xs: offset + b * xs + n] = torch.from_numpy(x2[b]).to(device)
     st = B.sysconv1d(xbuf.data_ptr() + 4 * offset, n, xs, np.ascontiguousarray(w_np), q,
                      ybuf.data_ptr() + 4 * offset, ys, batch, B.F32, design,
                      torch.cuda.current_stream().cuda_stream)
     assert st == 0, B.status_string(st)
     torch.cuda.synchronize()
     yh = ybuf.cpu().numpy()
-    out = np.stack([yh[offset + b * ys: offset + b * ys + n_out] for b in range(batch)])
+    out = np.lib.stride_tricks.as_strided(yh[offset:], shape=(batch, n_out), strides=(4 * ys, 4)).copy()
     mask = np.ones(yh.shape, bool)
-    for b in range(batch):
-        mask[offset + b * ys: offset + b * ys + n_out] = False
+    np.lib.stride_tricks.as_strided(mask[offset:], shape=(batch, n_out), strides=(ys, 1))[...] = False
     assert (yh[mask] == CANARY).all(), "write outside the output range"
     return out[0] if x_np.ndim == 1 else out
 
@@ -209,6 +208,25 @@ def test_1d_tiny_signals_all_designs(cuda_device, design, q, c_out):
         y = run_1d(x, w, design, cuda_device, batch_stride=stride)
         y_ref, s_ref = tiles_reference(x, w)
         assert_close_f32(y, y_ref, s_ref, "%s q=%d C=%d batch=%d" % (_ids(design), q, c_out, batch))
+
+
+@pytest.mark.parametrize("design", ALL_DESIGNS, ids=_ids)
+@pytest.mark.parametrize("q,c_out", [(5, 16), (2, 16), (8, 9), (3, 30)])
+def test_1d_tiny_signals_dense_and_shifted_layouts(cuda_device, design, q, c_out):
+    """The tiny-signal kernels move densely packed batches as whole 128-bit words and fall back to a gather for any
+    other layout: packed batches of several sizes (whole passes, a ragged last pass, fewer signals than one pass),
+    the same batches starting 1, 2 and 3 elements off a 16-byte boundary, and a stride one element longer."""
+    n = c_out + q - 1
+    rng = np.random.default_rng(4000 + 10 * q + c_out)
+    w = (rng.random(q, dtype=np.float32) * 2 - 1).astype(np.float32)
+    for batch in (3, 64, 257, 1536, 5001):
+        x = (rng.random((batch, n), dtype=np.float32) * 2 - 1).astype(np.float32)
+        y_ref, s_ref = tiles_reference(x, w)
+        for offset, stride in ((0, None), (1, None), (2, None), (3, None), (0, n + 1)):
+            y = run_1d(x, w, design, cuda_device, batch_stride=stride, offset=offset)
+            assert_close_f32(y, y_ref, s_ref, "%s q=%d C=%d batch=%d offset=%d stride=%s"
+                             % (_ids(design), q, c_out, batch, offset, stride))
+    assert B.device_status() == 0
 
 
 @pytest.mark.parametrize("design", ALL_DESIGNS, ids=_ids)
