@@ -361,6 +361,139 @@ conv2d_u8_is_dp4a_kernel(const Conv2DArgs a, const __grid_constant__ TapsPacked 
     }
 }
 
+// Input-stationary form that rebuilds the shifted words (filters of 8 to 15 rows, and of up to 4).  The kernel above
+// keeps the four shifted words of every stationary row in registers (8 P of them) and unrolls the row loop P
+// times; beyond seven rows neither fits, and for very short filters those registers cost more than they save.  Here a
+// word-PE keeps only each row's word and its right neighbour's word (4 P registers for the lane's two word-PEs), the
+// window slides by register moves, and the shifted words are rebuilt (PRMT) when they are used -- once per shift and
+// row, shared by the ceil(Q/4) tap groups: for one shift the products of all tap groups are summed first
+// (A_g = sum_p dp4a(x_p, w(p, g))), then the sums take their way up the word-PEs, z = shuffle(z) + A_g (integer
+// addition is exact in any order).  Geometry, loads and stores are those of the kernel above.
+template <int P, int Q>
+__global__ void __launch_bounds__(kThreads2)
+conv2d_u8_is_dp4a_rebuild_kernel(const Conv2DArgs a, const __grid_constant__ TapsPacked taps, const int band_h)
+{
+    dependent_launch_enter();
+    constexpr int G = IsDp4aGeom<Q>::G;
+    constexpr int kValid = IsDp4aGeom<Q>::kValid;
+    const int lane = threadIdx.x & (kLanes - 1);
+    const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;
+    const int c0 = strip * kValid;
+    const int r0 = blockIdx.y * band_h;
+    const int r1 = min(r0 + band_h, a.out_h);
+    const uint8_t *xb = static_cast<const uint8_t *>(a.x) + blockIdx.z * a.x_bstride;
+    int *yb = static_cast<int *>(a.y) + blockIdx.z * a.y_bstride;
+    if (c0 >= a.out_w) return;
+    const int y_align = row_alignment(static_cast<const int *>(a.y), a.y_pitch, a.y_bstride, a.batch);
+    const int oend = min(a.out_w, c0 + kValid);
+
+    bool ld_whole[2], ld_ragged[2], st_vec[2], st_part[2];
+#pragma unroll
+    for (int n = 0; n < 2; ++n) {
+        const int c = c0 + 4 * (kLanes * n + lane);
+        ld_whole[n] = c + 4 <= a.width;
+        ld_ragged[n] = !ld_whole[n] && c < a.width;
+        const int k = kLanes * n + lane - (G - 1);              // word-PE whose outputs end up here
+        st_vec[n] = k >= 0 && y_align == 4 && c0 + 4 * k + 4 <= oend;
+        st_part[n] = k >= 0 && !st_vec[n] && c0 + 4 * k < oend;
+    }
+    const uint8_t *xnext = xb + static_cast<long long>(r0) * a.x_pitch + c0 + 4 * lane;
+    int *onext = yb + static_cast<long long>(r0) * a.y_pitch + c0 + 4 * (lane - (G - 1));
+
+    auto fetch = [&](unsigned (&w)[2]) {
+#pragma unroll
+        for (int n = 0; n < 2; ++n) {
+            unsigned v = 0;
+            if (ld_whole[n]) {
+                v = __ldg(reinterpret_cast<const unsigned *>(xnext + 4 * kLanes * n));
+            } else if (ld_ragged[n]) {
+                const int c = c0 + 4 * (kLanes * n + lane);
+#pragma unroll
+                for (int e = 0; e < 3; ++e)
+                    if (c + e < a.width) v |= static_cast<unsigned>(xnext[4 * kLanes * n + e]) << (8 * e);
+            }
+            w[n] = v;
+        }
+        xnext += a.x_pitch;
+    };
+    // the next PE's words: the next lane's, and for lane 31 of run 0 the first word of run 1
+    auto neighbours = [&](const unsigned (&w)[2], unsigned (&nx)[2]) {
+        const unsigned send = lane == 0 ? w[1] : w[0];
+        nx[0] = __shfl_sync(kFullMask, send, (lane + 1) & (kLanes - 1));
+        nx[1] = __shfl_down_sync(kFullMask, w[1], 1);           // the strip's last PE keeps its own: invalid sums
+    };
+
+    // PE registers: the window of P input rows, each as the PE's word and its right neighbour's word
+    unsigned W[P][2], N[P][2];
+#pragma unroll
+    for (int p = 0; p < P; ++p)
+#pragma unroll
+        for (int n = 0; n < 2; ++n) W[p][n] = N[p][n] = 0;
+#pragma unroll
+    for (int p = 1; p < P; ++p) fetch(W[p]);    // rows r0 .. r0+P-2 sit one slot low: the first slide moves them up
+#pragma unroll
+    for (int p = 1; p < P; ++p) neighbours(W[p], N[p]);         // (after all the loads: they are in flight together)
+    unsigned nW[2] = {0u, 0u};
+    fetch(nW);
+
+#pragma unroll 1
+    for (int r = r0; r < r1; ++r) {
+        // the window slides down one row
+#pragma unroll
+        for (int p = 0; p < P - 1; ++p)
+#pragma unroll
+            for (int n = 0; n < 2; ++n) {
+                W[p][n] = W[p + 1][n];
+                N[p][n] = N[p + 1][n];
+            }
+        W[P - 1][0] = nW[0];
+        W[P - 1][1] = nW[1];
+        neighbours(nW, N[P - 1]);
+        if (r + 1 < r1) fetch(nW);
+
+        int Z[2][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            // products of every tap group with the inputs shifted by i pixels
+            int A[G][2];
+#pragma unroll
+            for (int g = 0; g < G; ++g) A[g][0] = A[g][1] = 0;
+#pragma unroll
+            for (int p = 0; p < P; ++p) {
+#pragma unroll
+                for (int n = 0; n < 2; ++n) {
+                    const unsigned sw = i == 0 ? W[p][n]
+                                               : __byte_perm(W[p][n], N[p][n], i == 1 ? 0x4321 : i == 2 ? 0x5432 : 0x6543);
+#pragma unroll
+                    for (int g = 0; g < G; ++g) A[g][n] = dp4a_u8s8(sw, taps.w[p * 4 + g], A[g][n]);
+                }
+            }
+            // the sums move one word-PE up per tap group: run 0 from the previous lane, run 1 likewise, its first PE
+            // from the last PE of run 0 (the strip's first PE has no left neighbour: invalid sums)
+            int z0 = A[0][0], z1 = A[0][1];
+#pragma unroll
+            for (int g = 1; g < G; ++g) {
+                const int send = lane == kLanes - 1 ? z0 : z1;
+                const int u0 = __shfl_up_sync(kFullMask, z0, 1);
+                const int u1 = __shfl_sync(kFullMask, send, (lane - 1) & (kLanes - 1));
+                z0 = u0 + A[g][0];
+                z1 = u1 + A[g][1];
+            }
+            Z[0][i] = z0;
+            Z[1][i] = z1;
+        }
+#pragma unroll
+        for (int n = 0; n < 2; ++n) {
+            if (st_vec[n])
+                *reinterpret_cast<int4 *>(onext + 4 * kLanes * n) = make_int4(Z[n][0], Z[n][1], Z[n][2], Z[n][3]);
+            else if (st_part[n])
+                store_group<U8Traits>(onext - (c0 + 4 * (lane - (G - 1))), c0 + 4 * (kLanes * n + lane - (G - 1)), oend,
+                                      y_align, Z[n]);
+        }
+        onext += a.y_pitch;
+    }
+}
+
 template <int P, int Q>
 cudaError_t launch_conv2d_u8_is_dp4a(const Conv2DArgs &a, const Taps2DInt &t, cudaStream_t s)
 {
@@ -385,13 +518,21 @@ cudaError_t launch_conv2d_u8_is_dp4a(const Conv2DArgs &a, const Taps2DInt &t, cu
     const long long fit = (a.out_h + 65534LL) / 65535;  // grid.y limit
     if (h < fit) h = fit;
     int band_h = static_cast<int>(h);
+    // which form: the ring of expanded rows pays for 5 to 7 filter rows (3840 x 2160, 7x7: 16.3 against 16.9 us);
+    // with fewer rows rebuilding the shifted words costs less than the ring's registers (3x3: 9.4 against 11.8 us),
+    // with more rows the ring does not fit
+    constexpr bool kRebuild = P <= 4 || P > 7;
     {
-        static const long long slots = 148LL * resident_blocks_per_sm(conv2d_u8_is_dp4a_kernel<P, Q>, kThreads2);
+        static const long long slots = 148LL * [] {
+            if constexpr (kRebuild) return resident_blocks_per_sm(conv2d_u8_is_dp4a_rebuild_kernel<P, Q>, kThreads2);
+            else return resident_blocks_per_sm(conv2d_u8_is_dp4a_kernel<P, Q>, kThreads2);
+        }();
         const long long per_band = static_cast<long long>((strips + kWarps2 - 1) / kWarps2) * a.batch;
         if (small_problem(a.out_h, per_band, 4, slots)) band_h = pick_band_height_small(a.out_h, per_band, P, 4, 64, slots);
     }
     dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + band_h - 1) / band_h, a.batch);
-    launch_kernel(conv2d_u8_is_dp4a_kernel<P, Q>, grid, kThreads2, s, a, pk, band_h);
+    if constexpr (kRebuild) launch_kernel(conv2d_u8_is_dp4a_rebuild_kernel<P, Q>, grid, kThreads2, s, a, pk, band_h);
+    else launch_kernel(conv2d_u8_is_dp4a_kernel<P, Q>, grid, kThreads2, s, a, pk, band_h);
     return cudaGetLastError();
 }
 
@@ -399,13 +540,9 @@ template <int P, int Q>
 struct FastPath2D<U8Traits, SYSCONV_IS, P, Q> {
     static bool launch(const Conv2DArgs &a, const Taps2DInt &taps, cudaStream_t s, cudaError_t *err)
     {
-        if constexpr (P <= 7) {
-            if (!u8_dp4a_eligible(a)) return false;
-            *err = launch_conv2d_u8_is_dp4a<P, Q>(a, taps, s);
-            return true;
-        } else {
-            return false;
-        }
+        if (!u8_dp4a_eligible(a)) return false;
+        *err = launch_conv2d_u8_is_dp4a<P, Q>(a, taps, s);
+        return true;
     }
 };
 

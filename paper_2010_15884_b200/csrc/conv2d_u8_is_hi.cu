@@ -1,5 +1,5 @@
 // 2-D uint8 x int8 -> int32 kernels of the input-stationary (SBM) design, filter heights 11..15 (all widths 1..15).
-#include "conv2d_kernels.cuh"
+#include "conv2d_u8_dp4a.cuh"
 
 namespace sysconv {
 

@@ -1204,8 +1204,8 @@ def test_2d_u8_shapes_and_extremes(cuda_device, design, pq):
 @pytest.mark.parametrize("pq", [(1, 1), (3, 3), (5, 5), (7, 7), (7, 15), (8, 15), (15, 15), (9, 2), (4, 13), (12, 8),
                                 (1, 4), (2, 5), (6, 9), (7, 12), (3, 8)], ids=lambda f: "%dx%d" % f)
 def test_2d_u8_packed_rows(cuda_device, design, pq):
-    """Rows that start 4-byte aligned take the packed four-taps-per-step kernels (OS: every filter size; IS: up to
-    seven filter rows; WS: rows aligned to 16 bytes): several strips, a ragged right edge, pitch padding, unaligned
+    """Rows that start 4-byte aligned take the packed four-taps-per-step kernels (OS and IS: every filter size, IS in
+    two forms by filter height; WS: rows aligned to 16 bytes): several strips, a ragged right edge, pitch padding, unaligned
     outputs, and the extreme pixel/tap values."""
     p, q = pq
     x, ws = inputs.gen_2d_u8s8(1101, 41, [pq], seed=90 + p + q, batch=2)
