@@ -227,7 +227,8 @@ def conv2d_separable(x, u, v, out=None, stream=None):
     v = np.ascontiguousarray(v, dtype=np.float32).reshape(-1)
     batch, h, wd = x3.shape
     if out is None:
-        out = torch.empty((batch, max(h - len(u) + 1, 0), max(wd - len(v) + 1, 0)), dtype=torch.float32, device=x.device)
+        ow = max(wd - len(v) + 1, 0)             # rows padded to 16 bytes, as in conv2d
+        out = torch.empty((batch, max(h - len(u) + 1, 0), (ow + 3) // 4 * 4), dtype=torch.float32, device=x.device)[:, :, :ow]
     y3 = out.unsqueeze(0) if out.dim() == 2 else out
     st = sysconv2d_separable(x3.data_ptr(), wd, h, x3.stride(1), x3.stride(0) if batch > 1 else 0, u, v, y3.data_ptr(),
                              y3.stride(1), y3.stride(0) if batch > 1 else 0, batch, _stream_ptr(stream))
@@ -427,7 +428,10 @@ def stencil2d(u, k, sweeps, out=None, scratch=None, stream=None):
 
 
 def conv2d(x, w, design=OS, out=None, stream=None, stride=1):
-    """y[b, r, c] = sum_p sum_q w[p, q] x[b, stride*r+p, stride*c+q] on CUDA tensors. x: (h, w) or (batch, h, w)."""
+    """y[b, r, c] = sum_p sum_q w[p, q] x[b, stride*r+p, stride*c+q] on CUDA tensors. x: (h, w) or (batch, h, w).
+
+    Without `out` the result is a view of a buffer whose rows are padded to 16 bytes (rows that start unaligned
+    are stored element by element, about twice as slow for the memory-bound filters)."""
     import torch
     if not x.is_cuda:
         raise SysconvError(-1, "conv2d (x is not a CUDA tensor; there is no CPU path)")
@@ -442,7 +446,9 @@ def conv2d(x, w, design=OS, out=None, stream=None, stride=1):
     if out is None:
         oh = (h - p) // stride + 1 if h >= p else 0
         ow = (wd - q) // stride + 1 if wd >= q else 0
-        out = torch.empty((batch, oh, ow), dtype=out_dtype, device=x.device)
+        # rows padded to a multiple of four elements (16 bytes) so that every row leaves as 128-bit stores; the
+        # result is the (batch, oh, ow) view of that buffer (call .contiguous() for a packed copy)
+        out = torch.empty((batch, oh, (ow + 3) // 4 * 4), dtype=out_dtype, device=x.device)[:, :, :ow]
         y3 = out
     else:
         y3 = out.unsqueeze(0) if out.dim() == 2 else out

@@ -1,4 +1,5 @@
-// 2-D fp32 weight-stationary convolution for the small filters (at most 8 filter columns, P*Q <= 32): the arrays
+// 2-D fp32 weight-stationary convolution for the smaller filters (at most 8 filter columns, window of at most 96
+// registers: up to 9 x 8 and 15 x 4): the arrays
 // side by side ALONG THE ROWS, everything in registers, no shared memory.
 //
 // As in the other weight-stationary kernels an array (Q PEs, PE q keeps the P taps of filter column q) is folded
@@ -28,7 +29,9 @@ constexpr int kWsrWarps = 4;
 template <int P, int Q>
 struct WsrShape {
     static constexpr int kSeg = Q <= 4 ? 4 : 8;                 // image columns per array and pass
-    static constexpr bool kFits = Q <= 8 && (P + kWsrM - 1) * kSeg <= 64;
+    // window registers: (P+3) x segment.  Measured on 2 x 2048 x 4096 against the form with transposed staging: 6x5
+    // 65 -> 37 us, 7x7 72 -> 50, 8x6 73 -> 52, 9x7 79 -> 70, 9x8 level; 11 rows: 11x5 76 -> 66 but 11x8 86 -> 104
+    static constexpr bool kFits = Q <= 8 && (P + kWsrM - 1) * kSeg <= 96;
     static constexpr int kOut = (kLanes - 1) * kSeg;            // output columns per warp
 };
 

@@ -530,6 +530,19 @@ BAD_PIXELS = ((0, 0, np.inf), (40, 127, np.nan), (41, 128, -np.inf), (63, 255, n
               (119, 299, np.inf), (100, 5, np.inf))
 
 
+@pytest.mark.parametrize("pq", [(6, 5), (7, 8), (8, 7), (9, 8), (9, 5), (15, 4), (14, 3), (11, 4), (13, 2)],
+                         ids=lambda f: "%dx%d" % f)
+def test_2d_ws_register_form_taller_filters(cuda_device, pq):
+    """The all-register weight-stationary form takes every filter of at most 8 columns whose window of P+3 rows fits
+    96 registers: several slices of 31 segments, a ragged last slice, bands that end inside a four-row pass, a batch,
+    and rows that do not start 16-byte aligned."""
+    p, q = pq
+    x, ws = inputs.gen_2d_f32(1030, 90, [pq], seed=700 + 16 * p + q, batch=2)
+    check_2d(x, ws[pq], B.WS, cuda_device)
+    check_2d(x[:, :67, :517], ws[pq], B.WS, cuda_device, x_pitch=519, y_pitch=517)
+    assert B.device_status() == 0
+
+
 @pytest.mark.parametrize("design", DESIGNS, ids=_ids)
 @pytest.mark.parametrize("pq", [(3, 3), (5, 5), (8, 6), (9, 9), (10, 7), (15, 15), (4, 8), (12, 12)],
                          ids=lambda f: "%dx%d" % f)
