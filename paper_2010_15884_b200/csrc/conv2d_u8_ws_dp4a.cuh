@@ -26,7 +26,6 @@ constexpr int kU8WsWarps = 4;
 constexpr int kU8WsSeg = 16;                    // pixels per array and pass (one 128-bit load)
 constexpr int kU8WsOut = (kLanes - 1) * kU8WsSeg;
 constexpr int kU8WsPitch = kU8WsSeg + 4;        // ints per lane block of the output staging row
-constexpr int kU8WsUnrollP = 7;                 // filters up to this height: every input row of a pass unrolled
 
 template <int P, int Q>
 __global__ void __launch_bounds__(kU8WsWarps *kLanes)
@@ -59,10 +58,8 @@ conv2d_u8_ws_dp4a_kernel(const Conv2DArgs a, const __grid_constant__ TapsPacked 
             for (int c = 0; c < SEG + TAIL; ++c) acc[m][c] = 0;
         // One input row: fetched once, its 16 shifted words built once, used by every output row it reaches.  FULL:
         // the row reaches all four output rows (kk in [M-1, P-1]), through the filter rows kk-m.
-        auto input_row = [&](auto full_tag, int kk) {
-            constexpr bool FULL = decltype(full_tag)::value;
+        auto load_row = [&](int kk, unsigned (&W)[5]) {
             const uint8_t *rowp = xb + static_cast<long long>(min(rg + kk, a.height - 1)) * a.x_pitch + col0;
-            unsigned W[5];
             if (whole) {
                 const uint4 t = __ldg(reinterpret_cast<const uint4 *>(rowp));
                 W[0] = t.x; W[1] = t.y; W[2] = t.z; W[3] = t.w;
@@ -76,6 +73,9 @@ conv2d_u8_ws_dp4a_kernel(const Conv2DArgs a, const __grid_constant__ TapsPacked 
                     W[j] = v;
                 }
             }
+        };
+        auto use_row = [&](auto full_tag, int kk, unsigned (&W)[5]) {
+            constexpr bool FULL = decltype(full_tag)::value;
             W[4] = __shfl_down_sync(kFullMask, W[0], 1);        // the first pixels of the next segment
             int wt[M][G];                                       // the taps through which this row reaches the four output rows
 #pragma unroll
@@ -96,17 +96,41 @@ conv2d_u8_ws_dp4a_kernel(const Conv2DArgs a, const __grid_constant__ TapsPacked 
                 }
             }
         };
-        if constexpr (P <= kU8WsUnrollP) {
+        // Short filters: every input row of a pass unrolled.  From five rows on the rows that reach all four output
+        // rows run in a loop (measured on 2 x 2048 x 4096: 7x13 90 -> 67 us, 5x13 71 -> 54, 7x7 44 -> 40; narrow
+        // filters of 5 to 7 rows are the exception: 7x3 36 -> 43 us, so they stay unrolled; from eight rows on the
+        // unrolled code also takes minutes to compile)
+        constexpr bool kRolled = P >= 8 || (P >= 5 && Q > 4);
+        if constexpr (!kRolled) {
 #pragma unroll
-            for (int kk = 0; kk < K; ++kk) input_row(std::false_type{}, kk);
+            for (int kk = 0; kk < K; ++kk) {
+                unsigned W[5];
+                load_row(kk, W);
+                use_row(std::false_type{}, kk, W);
+            }
         } else {
-            // tall filters: the rows that reach all four output rows run in a loop (code size), the others unrolled
+            // the rows that reach all four output rows run in a loop, the others unrolled; the next row is fetched
+            // before the current one is used
 #pragma unroll
-            for (int kk = 0; kk < M - 1; ++kk) input_row(std::false_type{}, kk);
+            for (int kk = 0; kk < M - 1; ++kk) {
+                unsigned W[5];
+                load_row(kk, W);
+                use_row(std::false_type{}, kk, W);
+            }
+            unsigned Wn[5];
+            load_row(M - 1, Wn);
 #pragma unroll 1
-            for (int kk = M - 1; kk < P; ++kk) input_row(std::true_type{}, kk);
+            for (int kk = M - 1; kk < P; ++kk) {
+                unsigned W[5] = {Wn[0], Wn[1], Wn[2], Wn[3], 0u};
+                load_row(kk + 1, Wn);
+                use_row(std::true_type{}, kk, W);
+            }
 #pragma unroll
-            for (int kk = P; kk < K; ++kk) input_row(std::false_type{}, kk);
+            for (int kk = P; kk < K; ++kk) {
+                unsigned W[5] = {Wn[0], Wn[1], Wn[2], Wn[3], 0u};
+                if (kk + 1 < K) load_row(kk + 1, Wn);
+                use_row(std::false_type{}, kk, W);
+            }
         }
         // the successor's share of this segment's last TAIL outputs comes back by shuffle
 #pragma unroll
