@@ -114,10 +114,11 @@ template <int P, int Q>
 cudaError_t launch_conv2d_sep_pq(const Conv2DArgs &a, const TapsSep &taps, cudaStream_t s)
 {
     if (a.batch > 65535) return cudaErrorInvalidConfiguration;
-    // eight PEs per lane and two rows in flight (the memory-bound shape) while the P partial rows fit the
-    // registers (P <= 11; measured 9+9: 0.487 -> 0.456 ms against four PEs); four PEs per lane for taller
+    // eight PEs per lane and two rows in flight (the memory-bound shape) while the P partial rows fit 128 registers
+    // (measured 9+9: 0.487 -> 0.456 ms against four PEs; 11 rows need 159 registers and ran 47-58 us on 2 x 2048 x 4096
+    // where 9 rows take 35-39, 10 rows with more than 9 columns 70-77 against 58); four PEs per lane for taller
     // filters and on small images
-    constexpr int RW = P <= 11 ? 8 : 4;
+    constexpr int RW = (P <= 9 || (P == 10 && Q <= 9)) ? 8 : 4;
     const long long strips8 = (a.out_w + 255) / 256;
     const bool narrow = RW == 8 && strips8 * a.batch * ((a.out_h + 7) / 8) < 148LL * 8 * 4;
     const int per_strip = narrow ? kLanes * 4 : kLanes * RW;
