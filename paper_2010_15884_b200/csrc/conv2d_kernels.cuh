@@ -759,6 +759,10 @@ cudaError_t launch_conv2d_pq(const Conv2DArgs &a, const typename Tr::taps_t &tap
         const long long strips8 = (a.out_w + 255) / 256;
         const long long warps8 = strips8 * a.batch * ((a.out_h + 7) / 8);
         if (warps8 < 148LL * 8 * 4) return launch_conv2d_osis<Tr, DESIGN, P, Q, 4>(a, taps, s);
+        // narrow image: 256-PE strips would stand idle for a quarter or more of what 128-PE strips cover
+        // (batches of short signals arrive here as images of a few dozen to a few hundred columns)
+        const long long cover8 = strips8 * 256, cover4 = (a.out_w + 127) / 128 * 128LL;
+        if (cover4 * 5 <= cover8 * 4) return launch_conv2d_osis<Tr, DESIGN, P, Q, 4>(a, taps, s);
     }
     return launch_conv2d_osis<Tr, DESIGN, P, Q, Sh::kR>(a, taps, s);
 }

@@ -217,6 +217,19 @@ int sysconv1d(const void *x_dev, long long n, long long x_batch_stride, const vo
         int launches = 0;
         // a batch of tiny signals (the paper's own experiment shape): small arrays side by side in a warp
         if (conv1d_tiles_eligible(a, design, q)) return finish(launch_conv1d_f32_tiles(design, a, w, q, s, &launches), launches);
+        // a batch of SHORT signals: the 1-D kernels give every signal tiles of 1216 or more outputs of its own, so
+        // signals of a few hundred samples would leave most of each array idle.  Such a batch is an image with one
+        // signal per row and a one-row filter: the 2-D kernels of the same design march down the rows with
+        // 128- or 256-PE strips (2^26 samples as signals of 100: 0.9-1.3 ms -> 0.13-0.33 ms; equal at 1000)
+        if (batch >= 2 && n_out <= kShortSignal1 && q <= kMaxQ2 && main_design(design)) {
+            Conv2DArgs g;
+            g.x = x_dev; g.y = y_dev;
+            g.width = static_cast<int>(n); g.height = batch;
+            g.out_w = static_cast<int>(n_out); g.out_h = batch;
+            g.x_pitch = x_batch_stride; g.y_pitch = y_batch_stride;
+            g.x_bstride = 0; g.y_bstride = 0; g.batch = 1;
+            return dispatch2d(g, w_host, q, 1, dtype, design, s);
+        }
         const DeviceInfo *d = device_info();
         if (!d) return SYSCONV_ECUDA;
         cudaError_t err = design == SYSCONV_OS   ? launch_conv1d_f32_os(a, w, q, d->status_word, s, &launches)
@@ -229,12 +242,13 @@ int sysconv1d(const void *x_dev, long long n, long long x_batch_stride, const vo
     if (!main_design(design)) return SYSCONV_EUNSUPPORTED;
     if (q > kMaxQ2) return SYSCONV_EUNSUPPORTED;
     if (n > 0x7fffffffLL) return SYSCONV_EUNSUPPORTED;
+    // one signal per image row (the batch stride is the row pitch)
     Conv2DArgs a;
     a.x = x_dev; a.y = y_dev;
-    a.width = static_cast<int>(n); a.height = 1;
-    a.out_w = static_cast<int>(n_out); a.out_h = 1;
-    a.x_pitch = n; a.y_pitch = n_out;
-    a.x_bstride = x_batch_stride; a.y_bstride = y_batch_stride; a.batch = batch;
+    a.width = static_cast<int>(n); a.height = batch;
+    a.out_w = static_cast<int>(n_out); a.out_h = batch;
+    a.x_pitch = x_batch_stride; a.y_pitch = y_batch_stride;
+    a.x_bstride = 0; a.y_bstride = 0; a.batch = 1;
     return dispatch2d(a, w_host, q, 1, dtype, design, s);
 }
 

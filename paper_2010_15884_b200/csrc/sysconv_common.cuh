@@ -26,6 +26,7 @@ constexpr int kMaxQ1 = 32;
 constexpr int R1 = 20;
 constexpr int kWarpIn1 = kLanes * R1;          // 640
 constexpr int kHalo1 = 32;
+constexpr int kShortSignal1 = 512;              // batches of signals with at most this many outputs run as images, one signal per row
 constexpr int kWarpOut1 = kWarpIn1 - kHalo1;   // 608
 // weight-stationary arrays, 1-D: one array per lane, each streaming a 76-output segment
 // (76 floats = 19 16-byte words: the lanes' 128-bit reads of their own segments fall in distinct banks)

@@ -1242,6 +1242,54 @@ def test_1d_u8(cuda_device, design):
     np.testing.assert_array_equal(y.cpu().numpy(), oracle.conv1d_u8s8_s32(x, ws[7]))
 
 
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+def test_1d_u8_batches(cuda_device, design):
+    """Integer signals run as images with one signal per row: a batch of short signals, packed and with a longer
+    stride, canaries between the outputs."""
+    rng = np.random.default_rng(77)
+    for n, batch, q, stride in ((300, 40, 7, None), (300, 40, 7, 304), (33, 1000, 4, 36), (5000, 3, 15, 5003)):
+        x = rng.integers(0, 256, (batch, n), dtype=np.uint8)
+        w = rng.integers(-128, 128, q, dtype=np.int8)
+        xs = stride or n
+        n_out = n - q + 1
+        ys = stride or n_out
+        xh = np.zeros(batch * xs + 16, np.uint8)
+        np.lib.stride_tricks.as_strided(xh, shape=(batch, n), strides=(xs, 1))[...] = x
+        xd = torch.from_numpy(xh).to(cuda_device)
+        yd = torch.full((batch * ys + 16,), 123456789, dtype=torch.int32, device=cuda_device)
+        st = B.sysconv1d(xd.data_ptr(), n, xs, w, q, yd.data_ptr(), ys, batch, B.U8S8_S32, design,
+                         torch.cuda.current_stream().cuda_stream)
+        assert st == 0, B.status_string(st)
+        torch.cuda.synchronize()
+        yh = yd.cpu().numpy()
+        got = np.lib.stride_tricks.as_strided(yh, shape=(batch, n_out), strides=(4 * ys, 4))
+        for b in range(0, batch, max(batch // 7, 1)):
+            np.testing.assert_array_equal(got[b], oracle.conv1d_u8s8_s32(x[b], w))
+        mask = np.ones(yh.shape, bool)
+        np.lib.stride_tricks.as_strided(mask, shape=(batch, n_out), strides=(ys, 1))[...] = False
+        assert (yh[mask] == 123456789).all(), "write outside the output range"
+    assert B.device_status() == 0
+
+
+@pytest.mark.parametrize("design", DESIGNS, ids=_ids)
+@pytest.mark.parametrize("q", [1, 4, 9, 15, 16])
+def test_1d_short_signal_batches(cuda_device, design, q):
+    """Batches of short signals (more than 32 and at most 512 outputs, filters up to 15 taps) run as images with one
+    signal per row; longer signals, longer filters and single signals stay on the 1-D kernels.  Both sides of each
+    limit, packed and padded strides (rows 16-byte aligned or not), element offsets, canaries around every output."""
+    rng = np.random.default_rng(8100 + q)
+    w = (rng.random(q, dtype=np.float32) * 2 - 1).astype(np.float32)
+    for n_out, batch in ((33, 700), (100, 257), (255, 64), (512, 9), (513, 9), (300, 1), (300, 2)):
+        n = n_out + q - 1
+        x = (rng.random((batch, n), dtype=np.float32) * 2 - 1).astype(np.float32)
+        y_ref, s_ref = tiles_reference(x, w)
+        for offset, stride in ((0, None), (0, (n + 3) // 4 * 4), (1, n + 1), (3, None)):
+            y = run_1d(x, w, design, cuda_device, batch_stride=stride, offset=offset).reshape(batch, n_out)
+            assert_close_f32(y, y_ref, s_ref, "%s q=%d n_out=%d batch=%d offset=%d stride=%s"
+                             % (_ids(design), q, n_out, batch, offset, stride))
+    assert B.device_status() == 0
+
+
 # ------------------------------------------------------------------------ host-buffer entry points
 
 
