@@ -48,7 +48,7 @@ conv2d_is_pair_kernel(const Conv2DArgs a, const __grid_constant__ Taps2D taps, c
     constexpr int R = R2;
     static_assert(R == 4 && Q >= 2, "four PEs per lane; a pair needs two filter columns");
     const int lane = threadIdx.x & (kLanes - 1);
-    const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;
+    const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;    // (a block of fewer warps is the only one of its row)
     const int c0 = strip * G::kValid;           // first output column = first input column (PE 0)
     if (c0 >= a.out_w) return;
     const int r0 = blockIdx.y * band_h;
@@ -161,12 +161,13 @@ cudaError_t launch_conv2d_is_pair(const Conv2DArgs &a, const Taps2D &taps, cudaS
     const int per_strip = IsPairGeom<Q>::kValid;
     const int strips = (a.out_w + per_strip - 1) / per_strip;
     const int band_h = pick_band_height(a.out_h, static_cast<long long>(strips) * a.batch, P, Q);
-    dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + band_h - 1) / band_h, a.batch);
+    const int wpb = block_warps(strips, kWarps2);
+    dim3 grid((strips + wpb - 1) / wpb, (a.out_h + band_h - 1) / band_h, a.batch);
     if (grid.y > 65535) return cudaErrorInvalidConfiguration;
     // two output rows per pass up to ten filter rows (measured: 9x9 0.96 -> 0.85 ms); beyond that the
     // second row's registers cost more than the shared tap reads save (15x15: 2.33 ms with one row, 2.63 with two)
     constexpr int ROWS = P <= 10 ? 2 : 1;
-    launch_kernel(conv2d_is_pair_kernel<P, Q, ROWS, ROWS == 2 ? 4 : 1>, grid, kThreads2, s, a, taps, tp, band_h);
+    launch_kernel(conv2d_is_pair_kernel<P, Q, ROWS, ROWS == 2 ? 4 : 1>, grid, wpb * kLanes, s, a, taps, tp, band_h);
     return cudaGetLastError();
 }
 

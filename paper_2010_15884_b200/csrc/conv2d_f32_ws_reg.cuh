@@ -46,7 +46,7 @@ conv2d_ws_reg_kernel(const Conv2DArgs a, const __grid_constant__ Taps2D taps, co
     constexpr int kTail = Q - Q % 2;            // outputs at the end of a segment whose sums are still in flight
     static_assert(Q <= SEG, "a filter row longer than a segment breaks the hand-over");
     const int lane = threadIdx.x & (kLanes - 1);
-    const int slice = blockIdx.x * kWsrWarps + threadIdx.x / kLanes;
+    const int slice = blockIdx.x * kWsrWarps + threadIdx.x / kLanes;    // (a block of fewer warps is the only one of its row)
     const int c0 = slice * WsrShape<P, Q>::kOut;        // first output column of the slice
     if (c0 >= a.out_w) return;
     const int col0 = c0 + lane * SEG;                   // first image column of this lane's segment
@@ -154,9 +154,11 @@ cudaError_t launch_conv2d_ws_reg(const Conv2DArgs &a, const Taps2D &taps, cudaSt
             tp.w[p * (Q + 1) + t] = make_float2(t < Q ? taps.w[p * Q + t] : 0.f, t >= 1 ? taps.w[p * Q + t - 1] : 0.f);
     constexpr int kOut = WsrShape<P, Q>::kOut;
     const int slices = (a.out_w + kOut - 1) / kOut;
-    const long long per_band = static_cast<long long>((slices + kWsrWarps - 1) / kWsrWarps) * a.batch;
+    const int wpb = block_warps(slices, kWsrWarps);
+    const long long per_band = static_cast<long long>((slices + wpb - 1) / wpb) * a.batch;
     // bands of four-row passes; every band re-reads the P-1 rows above it
-    static const long long slots = 148LL * resident_blocks_per_sm(conv2d_ws_reg_kernel<P, Q>, kWsrWarps * kLanes);
+    static const long long slots4 = 148LL * resident_blocks_per_sm(conv2d_ws_reg_kernel<P, Q>, kWsrWarps * kLanes);
+    const long long slots = slots4 * kWsrWarps / wpb;       // smaller blocks: as many more of them are resident
     long long band_h;
     if (small_problem(a.out_h, per_band, kWsrM, slots)) {
         band_h = pick_band_height_small(a.out_h, per_band, P, kWsrM, 64, slots);
@@ -167,8 +169,8 @@ cudaError_t launch_conv2d_ws_reg(const Conv2DArgs &a, const Taps2D &taps, cudaSt
     }
     band_h = (band_h + kWsrM - 1) / kWsrM * kWsrM;
     if ((a.out_h + band_h - 1) / band_h > 65535) band_h = ((a.out_h + 65534) / 65535 + kWsrM - 1) / kWsrM * kWsrM;
-    dim3 grid((slices + kWsrWarps - 1) / kWsrWarps, static_cast<unsigned>((a.out_h + band_h - 1) / band_h), a.batch);
-    launch_kernel(conv2d_ws_reg_kernel<P, Q>, grid, kWsrWarps * kLanes, s, a, taps, tp, static_cast<int>(band_h));
+    dim3 grid((slices + wpb - 1) / wpb, static_cast<unsigned>((a.out_h + band_h - 1) / band_h), a.batch);
+    launch_kernel(conv2d_ws_reg_kernel<P, Q>, grid, wpb * kLanes, s, a, taps, tp, static_cast<int>(band_h));
     return cudaGetLastError();
 }
 

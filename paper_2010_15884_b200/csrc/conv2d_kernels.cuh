@@ -134,7 +134,7 @@ conv2d_os_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t
     constexpr bool kHalo = Q > 1;
     constexpr bool kHaloChain = Q - 1 > 4;      // the halo spans more than one lane
     const int lane = threadIdx.x & (kLanes - 1);
-    const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;
+    const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;    // (a block of fewer warps is the only one of its row)
     const int c0 = strip * kStrip;
     const int r0 = blockIdx.y * band_h;
     const int r1 = min(r0 + band_h, a.out_h);
@@ -263,7 +263,7 @@ conv2d_os_rowpair_kernel(const Conv2DArgs a, const __grid_constant__ TapsRowPair
     constexpr bool kHaloChain = Q - 1 > 4;
     constexpr int kStrip = kLanes * R;
     const int lane = threadIdx.x & (kLanes - 1);
-    const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;
+    const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;    // (a block of fewer warps is the only one of its row)
     const int c0 = strip * kStrip;
     if (c0 >= a.out_w) return;
     const int r0 = blockIdx.y * band_h;
@@ -395,7 +395,7 @@ conv2d_is_kernel(const Conv2DArgs a, const __grid_constant__ typename Tr::taps_t
     constexpr bool kRing = kIsRing<P, Q, R>;
     constexpr int U = kRing ? P : 1;            // output rows per trip of the row loop
     const int lane = threadIdx.x & (kLanes - 1);
-    const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;
+    const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;    // (a block of fewer warps is the only one of its row)
     const int c0 = strip * kValid;              // first output column = first input column (PE 0)
     const int r0 = blockIdx.y * band_h;
     const int r1 = min(r0 + band_h, a.out_h);
@@ -673,23 +673,25 @@ cudaError_t launch_conv2d_osis(const Conv2DArgs &a, const typename Tr::taps_t &t
     const int per_strip = DESIGN == SYSCONV_OS ? kLanes * R : IsGeom<Q, R>::kValid;
     const int strips = (a.out_w + per_strip - 1) / per_strip;
     int band_h = pick_band_height(a.out_h, static_cast<long long>(strips) * a.batch, P, Q);
+    const int wpb = block_warps(strips, kWarps2);
     {
         // a problem of a few waves of blocks: short bands, chosen by the number of waves they give
-        static const long long slots = 148LL * [] {
+        static const long long slots4 = 148LL * [] {
             if constexpr (DESIGN == SYSCONV_OS)
                 return resident_blocks_per_sm(conv2d_os_kernel<Tr, P, Q, R, Sh::kMinCtas, Sh::kPrefetch>, kThreads2);
             else
                 return resident_blocks_per_sm(conv2d_is_kernel<Tr, P, Q, R, Sh::kMinCtas>, kThreads2);
         }();
-        const long long per_band = static_cast<long long>((strips + kWarps2 - 1) / kWarps2) * a.batch;
+        const long long slots = slots4 * kWarps2 / wpb;      // smaller blocks: as many more of them are resident
+        const long long per_band = static_cast<long long>((strips + wpb - 1) / wpb) * a.batch;
         if (small_problem(a.out_h, per_band, 4, slots)) band_h = pick_band_height_small(a.out_h, per_band, P, 4, 64, slots);
     }
-    dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + band_h - 1) / band_h, a.batch);
+    dim3 grid((strips + wpb - 1) / wpb, (a.out_h + band_h - 1) / band_h, a.batch);
     if (grid.y > 65535) return cudaErrorInvalidConfiguration;
     if constexpr (DESIGN == SYSCONV_OS)
-        launch_kernel(conv2d_os_kernel<Tr, P, Q, R, Sh::kMinCtas, Sh::kPrefetch>, grid, kThreads2, s, a, taps, band_h);
+        launch_kernel(conv2d_os_kernel<Tr, P, Q, R, Sh::kMinCtas, Sh::kPrefetch>, grid, wpb * kLanes, s, a, taps, band_h);
     else
-        launch_kernel(conv2d_is_kernel<Tr, P, Q, R, Sh::kMinCtas>, grid, kThreads2, s, a, taps, band_h);
+        launch_kernel(conv2d_is_kernel<Tr, P, Q, R, Sh::kMinCtas>, grid, wpb * kLanes, s, a, taps, band_h);
     return cudaGetLastError();
 }
 
@@ -711,9 +713,10 @@ cudaError_t launch_conv2d_os_rowpair(const Conv2DArgs &a, const float *w, cudaSt
         }
     const int strips = (a.out_w + kLanes * R - 1) / (kLanes * R);
     const int band_h = pick_band_height(a.out_h, static_cast<long long>(strips) * a.batch, P, Q);
-    dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + band_h - 1) / band_h, a.batch);
+    const int wpb = block_warps(strips, kWarps2);
+    dim3 grid((strips + wpb - 1) / wpb, (a.out_h + band_h - 1) / band_h, a.batch);
     if (grid.y > 65535) return cudaErrorInvalidConfiguration;
-    launch_kernel(conv2d_os_rowpair_kernel<P, Q, R, MINB, kRowPairExact<P>>, grid, kThreads2, s, a, t, band_h);
+    launch_kernel(conv2d_os_rowpair_kernel<P, Q, R, MINB, kRowPairExact<P>>, grid, wpb * kLanes, s, a, t, band_h);
     return cudaGetLastError();
 }
 

@@ -39,7 +39,7 @@ conv2d_u8_os_dp4a_kernel(const Conv2DArgs a, const __grid_constant__ TapsPacked 
     // A strip is NW runs of 32 words; lane l holds word l of every run, so that each load and each 128-bit
     // store of a warp covers one contiguous piece of the row.
     const int lane = threadIdx.x & (kLanes - 1);
-    const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;
+    const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;    // (a block of fewer warps is the only one of its row)
     const int c0 = strip * kStrip;
     const int r0 = blockIdx.y * band_h;
     const int r1 = min(r0 + band_h, a.out_h);
@@ -204,15 +204,17 @@ cudaError_t launch_conv2d_u8_os_dp4a(const Conv2DArgs &a, const Taps2DInt &t, cu
     const long long fit = (a.out_h + 65534LL) / 65535;     // grid.y limit
     if (h < fit) h = fit;
     int band_h = static_cast<int>(h);
+    const int wpb = block_warps(strips, kWarps2);
     {
         // a problem of a few waves of blocks: bands chosen by the number of waves they give
-        static const long long slots = 148LL * resident_blocks_per_sm(conv2d_u8_os_dp4a_kernel<P, Q, PX, PF>, kThreads2);
-        const long long per_band = static_cast<long long>((strips + kWarps2 - 1) / kWarps2) * a.batch;
+        static const long long slots4 = 148LL * resident_blocks_per_sm(conv2d_u8_os_dp4a_kernel<P, Q, PX, PF>, kThreads2);
+        const long long slots = slots4 * kWarps2 / wpb;     // smaller blocks: as many more of them are resident
+        const long long per_band = static_cast<long long>((strips + wpb - 1) / wpb) * a.batch;
         if (small_problem(a.out_h, per_band, 4, slots)) band_h = pick_band_height_small(a.out_h, per_band, P, 4, 64, slots);
     }
-    dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + band_h - 1) / band_h, a.batch);
+    dim3 grid((strips + wpb - 1) / wpb, (a.out_h + band_h - 1) / band_h, a.batch);
     if (grid.y > 65535) return cudaErrorInvalidConfiguration;
-    launch_kernel(conv2d_u8_os_dp4a_kernel<P, Q, PX, PF>, grid, kThreads2, s, a, pk, band_h);
+    launch_kernel(conv2d_u8_os_dp4a_kernel<P, Q, PX, PF>, grid, wpb * kLanes, s, a, pk, band_h);
     return cudaGetLastError();
 }
 
@@ -240,7 +242,7 @@ conv2d_u8_is_dp4a_kernel(const Conv2DArgs a, const __grid_constant__ TapsPacked 
     constexpr int G = IsDp4aGeom<Q>::G;
     constexpr int kValid = IsDp4aGeom<Q>::kValid;
     const int lane = threadIdx.x & (kLanes - 1);
-    const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;
+    const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;    // (a block of fewer warps is the only one of its row)
     const int c0 = strip * kValid;              // first output column = first input column of the strip
     const int r0 = blockIdx.y * band_h;
     const int r1 = min(r0 + band_h, a.out_h);
@@ -377,7 +379,7 @@ conv2d_u8_is_dp4a_rebuild_kernel(const Conv2DArgs a, const __grid_constant__ Tap
     constexpr int G = IsDp4aGeom<Q>::G;
     constexpr int kValid = IsDp4aGeom<Q>::kValid;
     const int lane = threadIdx.x & (kLanes - 1);
-    const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;
+    const int strip = blockIdx.x * kWarps2 + threadIdx.x / kLanes;    // (a block of fewer warps is the only one of its row)
     const int c0 = strip * kValid;
     const int r0 = blockIdx.y * band_h;
     const int r1 = min(r0 + band_h, a.out_h);
@@ -522,17 +524,19 @@ cudaError_t launch_conv2d_u8_is_dp4a(const Conv2DArgs &a, const Taps2DInt &t, cu
     // with fewer rows rebuilding the shifted words costs less than the ring's registers (3x3: 9.4 against 11.8 us),
     // with more rows the ring does not fit
     constexpr bool kRebuild = P <= 4 || P > 7;
+    const int wpb = block_warps(strips, kWarps2);
     {
-        static const long long slots = 148LL * [] {
+        static const long long slots4 = 148LL * [] {
             if constexpr (kRebuild) return resident_blocks_per_sm(conv2d_u8_is_dp4a_rebuild_kernel<P, Q>, kThreads2);
             else return resident_blocks_per_sm(conv2d_u8_is_dp4a_kernel<P, Q>, kThreads2);
         }();
-        const long long per_band = static_cast<long long>((strips + kWarps2 - 1) / kWarps2) * a.batch;
+        const long long slots = slots4 * kWarps2 / wpb;
+        const long long per_band = static_cast<long long>((strips + wpb - 1) / wpb) * a.batch;
         if (small_problem(a.out_h, per_band, 4, slots)) band_h = pick_band_height_small(a.out_h, per_band, P, 4, 64, slots);
     }
-    dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + band_h - 1) / band_h, a.batch);
-    if constexpr (kRebuild) launch_kernel(conv2d_u8_is_dp4a_rebuild_kernel<P, Q>, grid, kThreads2, s, a, pk, band_h);
-    else launch_kernel(conv2d_u8_is_dp4a_kernel<P, Q>, grid, kThreads2, s, a, pk, band_h);
+    dim3 grid((strips + wpb - 1) / wpb, (a.out_h + band_h - 1) / band_h, a.batch);
+    if constexpr (kRebuild) launch_kernel(conv2d_u8_is_dp4a_rebuild_kernel<P, Q>, grid, wpb * kLanes, s, a, pk, band_h);
+    else launch_kernel(conv2d_u8_is_dp4a_kernel<P, Q>, grid, wpb * kLanes, s, a, pk, band_h);
     return cudaGetLastError();
 }
 

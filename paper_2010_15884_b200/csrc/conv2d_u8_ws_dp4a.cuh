@@ -34,7 +34,7 @@ conv2d_u8_ws_dp4a_kernel(const Conv2DArgs a, const __grid_constant__ TapsPacked 
     dependent_launch_enter();
     constexpr int M = kU8WsM, K = M + P - 1, G = (Q + 3) / 4, SEG = kU8WsSeg, TAIL = 4 * (G - 1);
     const int lane = threadIdx.x & (kLanes - 1);
-    const int slice = blockIdx.x * kU8WsWarps + threadIdx.x / kLanes;
+    const int slice = blockIdx.x * kU8WsWarps + threadIdx.x / kLanes;    // (a block of fewer warps is the only one of its row)
     const int c0 = slice * kU8WsOut;                    // first output column of the slice
     if (c0 >= a.out_w) return;
     const int col0 = c0 + lane * SEG;                   // first pixel of this lane's segment
@@ -185,8 +185,10 @@ cudaError_t launch_conv2d_u8_ws_dp4a(const Conv2DArgs &a, const Taps2DInt &t, cu
             pk.w[p * 4 + g] = static_cast<int>(v);
         }
     const int slices = (a.out_w + kU8WsOut - 1) / kU8WsOut;
-    const long long per_band = static_cast<long long>((slices + kU8WsWarps - 1) / kU8WsWarps) * a.batch;
-    static const long long slots = 148LL * resident_blocks_per_sm(conv2d_u8_ws_dp4a_kernel<P, Q>, kU8WsWarps * kLanes);
+    const int wpb = block_warps(slices, kU8WsWarps);
+    const long long per_band = static_cast<long long>((slices + wpb - 1) / wpb) * a.batch;
+    static const long long slots4 = 148LL * resident_blocks_per_sm(conv2d_u8_ws_dp4a_kernel<P, Q>, kU8WsWarps * kLanes);
+    const long long slots = slots4 * kU8WsWarps / wpb;      // smaller blocks: as many more of them are resident
     long long band_h;
     if (small_problem(a.out_h, per_band, kU8WsM, slots)) {
         band_h = pick_band_height_small(a.out_h, per_band, P, kU8WsM, 64, slots);
@@ -197,8 +199,8 @@ cudaError_t launch_conv2d_u8_ws_dp4a(const Conv2DArgs &a, const Taps2DInt &t, cu
     }
     band_h = (band_h + kU8WsM - 1) / kU8WsM * kU8WsM;
     if ((a.out_h + band_h - 1) / band_h > 65535) band_h = ((a.out_h + 65534) / 65535 + kU8WsM - 1) / kU8WsM * kU8WsM;
-    dim3 grid((slices + kU8WsWarps - 1) / kU8WsWarps, static_cast<unsigned>((a.out_h + band_h - 1) / band_h), a.batch);
-    launch_kernel(conv2d_u8_ws_dp4a_kernel<P, Q>, grid, kU8WsWarps * kLanes, s, a, pk, static_cast<int>(band_h));
+    dim3 grid((slices + wpb - 1) / wpb, static_cast<unsigned>((a.out_h + band_h - 1) / band_h), a.batch);
+    launch_kernel(conv2d_u8_ws_dp4a_kernel<P, Q>, grid, wpb * kLanes, s, a, pk, static_cast<int>(band_h));
     return cudaGetLastError();
 }
 

@@ -191,6 +191,15 @@ inline bool small_problem(int out_h, long long per_band, int lo, long long slots
     return per_band * ((out_h + lo - 1) / lo) <= 4 * slots;
 }
 
+// Warps per block of the 2-D kernels whose warps take neighbouring column strips: `full` of them, fewer when the image
+// has fewer strips -- the spare warps of a block would return at once and leave their share of the SM idle (narrow
+// images; batches of short signals, which arrive as images of a few dozen to a few hundred columns).  Such a block is
+// the only one of its row of the grid, so the kernels keep computing strip = blockIdx.x * full + warp.
+inline int block_warps(long long strips, int full)
+{
+    return strips >= full ? full : (strips < 1 ? 1 : static_cast<int>(strips));
+}
+
 // Sentinel returned by a launcher for a filter size it has no instantiation for.
 constexpr cudaError_t kNoInstantiation = cudaErrorInvalidKernelImage;
 
