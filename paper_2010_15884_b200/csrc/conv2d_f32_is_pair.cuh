@@ -151,12 +151,13 @@ conv2d_is_pair_kernel(const Conv2DArgs a, const __grid_constant__ Taps2D taps, c
 template <int P, int Q>
 cudaError_t launch_conv2d_is_pair(const Conv2DArgs &a, const Taps2D &taps, cudaStream_t s)
 {
+    static_assert(P * (Q + 1) <= kMaxP2 * (kMaxQ2 + 1), "tap-pair table too small");
     TapsColPairs tp{};
-    for (int p = 0; p < kMaxP2; ++p)
-        for (int t = 0; t <= kMaxQ2; ++t) {
-            const float cur = (p < P && t < Q) ? taps.w[p * Q + t] : 0.f;
-            const float prev = (p < P && t >= 1 && t <= Q) ? taps.w[p * Q + t - 1] : 0.f;
-            if (p < P && t <= Q) tp.w[p * (Q + 1) + t] = make_float2(cur, prev);
+    for (int p = 0; p < P; ++p)
+        for (int t = 0; t <= Q; ++t) {
+            const float cur = t < Q ? taps.w[p * Q + t] : 0.f;
+            const float prev = t >= 1 ? taps.w[p * Q + t - 1] : 0.f;
+            tp.w[p * (Q + 1) + t] = make_float2(cur, prev);
         }
     const int per_strip = IsPairGeom<Q>::kValid;
     const int strips = (a.out_w + per_strip - 1) / per_strip;

@@ -221,13 +221,16 @@ int sysconv1d(const void *x_dev, long long n, long long x_batch_stride, const vo
         // signals of a few hundred samples would leave most of each array idle.  Such a batch is an image with one
         // signal per row and a one-row filter: the 2-D kernels of the same design march down the rows with
         // 128- or 256-PE strips (2^26 samples as signals of 100: 0.9-1.3 ms -> 0.13-0.33 ms; equal at 1000)
-        if (batch >= 2 && n_out <= kShortSignal1 && q <= kMaxQ2 && main_design(design)) {
+        // Filters of 16 to 32 taps: the output- and input-stationary 2-D kernels are compiled for such rows as well.
+        const bool long_row = q > kMaxQ2 && (design == SYSCONV_OS || design == SYSCONV_IS);
+        if (batch >= 2 && n_out <= kShortSignal1 && main_design(design) && (q <= kMaxQ2 || long_row)) {
             Conv2DArgs g;
             g.x = x_dev; g.y = y_dev;
             g.width = static_cast<int>(n); g.height = batch;
             g.out_w = static_cast<int>(n_out); g.out_h = batch;
             g.x_pitch = x_batch_stride; g.y_pitch = y_batch_stride;
             g.x_bstride = 0; g.y_bstride = 0; g.batch = 1;
+            if (long_row) return finish(launch_conv2d_f32_long_rows(design, g, w, q, s, &launches), launches);
             return dispatch2d(g, w_host, q, 1, dtype, design, s);
         }
         const DeviceInfo *d = device_info();

@@ -103,6 +103,7 @@ cudaError_t launch_conv2d_f32_separable(const Conv2DArgs &a, const float *u, int
                                         int *launches);
 
 // iterated 3x3 stencil (stencil2d_f32.cu): `fused` sweeps (1..4) in one launch; a.out_w/out_h unused (output = grid size)
+cudaError_t launch_conv2d_f32_long_rows(int design, const Conv2DArgs &a, const float *w, int q, cudaStream_t s, int *launches);
 cudaError_t launch_stencil2d_f32(const Conv2DArgs &a, const float *k9, int fused, cudaStream_t s, int *launches);
 
 // generic space-time executor (spacetime.cu): *status receives the planning result

@@ -1272,10 +1272,10 @@ def test_1d_u8_batches(cuda_device, design):
 
 
 @pytest.mark.parametrize("design", DESIGNS, ids=_ids)
-@pytest.mark.parametrize("q", [1, 4, 9, 15, 16])
+@pytest.mark.parametrize("q", [1, 4, 9, 15, 16, 23, 32])
 def test_1d_short_signal_batches(cuda_device, design, q):
-    """Batches of short signals (more than 32 and at most 512 outputs, filters up to 15 taps) run as images with one
-    signal per row; longer signals, longer filters and single signals stay on the 1-D kernels.  Both sides of each
+    """Batches of short signals (more than 32 and at most 512 outputs) run as images with one signal per row (filters
+    of more than 15 taps: output- and input-stationary only); longer signals and single signals stay on the 1-D kernels.  Both sides of each
     limit, packed and padded strides (rows 16-byte aligned or not), element offsets, canaries around every output."""
     rng = np.random.default_rng(8100 + q)
     w = (rng.random(q, dtype=np.float32) * 2 - 1).astype(np.float32)
