@@ -124,9 +124,10 @@ cudaError_t launch_conv2d_sep_pq(const Conv2DArgs &a, const TapsSep &taps, cudaS
     const int per_strip = narrow ? kLanes * 4 : kLanes * RW;
     const int strips = (a.out_w + per_strip - 1) / per_strip;
     const int band_h = pick_band_height(a.out_h, static_cast<long long>(strips) * a.batch, P, 1);
-    dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + band_h - 1) / band_h, a.batch);
-    if (narrow) launch_kernel(conv2d_sep_os_kernel<P, Q, 4, 2>, grid, kThreads2, s, a, taps, band_h);
-    else launch_kernel(conv2d_sep_os_kernel<P, Q, RW, 2>, grid, kThreads2, s, a, taps, band_h);
+    const int wpb = block_warps(strips, kWarps2);       // narrow images: blocks of as many warps as there are strips
+    dim3 grid((strips + wpb - 1) / wpb, (a.out_h + band_h - 1) / band_h, a.batch);
+    if (narrow) launch_kernel(conv2d_sep_os_kernel<P, Q, 4, 2>, grid, wpb * kLanes, s, a, taps, band_h);
+    else launch_kernel(conv2d_sep_os_kernel<P, Q, RW, 2>, grid, wpb * kLanes, s, a, taps, band_h);
     return cudaGetLastError();
 }
 

@@ -211,9 +211,10 @@ cudaError_t launch_conv2d_s2_pq(const Conv2DArgs &a, const Taps2D &taps, cudaStr
     const int per_strip = DESIGN == SYSCONV_OS ? kStripOutS2 : IsGeomS2<Q>::kValid;
     const int strips = (a.out_w + per_strip - 1) / per_strip;
     const int band_h = pick_band_height(a.out_h, static_cast<long long>(strips) * a.batch, P, Q);
-    dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.out_h + band_h - 1) / band_h, a.batch);
-    if (DESIGN == SYSCONV_OS) launch_kernel(conv2d_os_s2_kernel<P, Q>, grid, kThreads2, s, a, taps, band_h);
-    else launch_kernel(conv2d_is_s2_kernel<P, Q>, grid, kThreads2, s, a, taps, band_h);
+    const int wpb = block_warps(strips, kWarps2);       // narrow images: blocks of as many warps as there are strips
+    dim3 grid((strips + wpb - 1) / wpb, (a.out_h + band_h - 1) / band_h, a.batch);
+    if (DESIGN == SYSCONV_OS) launch_kernel(conv2d_os_s2_kernel<P, Q>, grid, wpb * kLanes, s, a, taps, band_h);
+    else launch_kernel(conv2d_is_s2_kernel<P, Q>, grid, wpb * kLanes, s, a, taps, band_h);
     return cudaGetLastError();
 }
 

@@ -174,16 +174,18 @@ cudaError_t launch_stencil2d_t(const Conv2DArgs &a, const StencilCoef &coef, boo
 {
     constexpr int V = StencilGeom<T>::kValid;
     const int strips = (a.width + V - 1) / V;
-    const long long per_band = static_cast<long long>((strips + kWarps2 - 1) / kWarps2) * a.batch;
+    const int wpb = block_warps(strips, kWarps2);       // narrow grids: blocks of as many warps as there are strips
+    const long long per_band = static_cast<long long>((strips + wpb - 1) / wpb) * a.batch;
     // bands re-read and re-compute 2T rows each: long bands for large grids, bands by the number of block waves
     // for small ones
     int band_h = 128;
-    static const long long slots = 148LL * resident_blocks_per_sm(stencil2d_kernel<T, false>, kThreads2);
+    static const long long slots4 = 148LL * resident_blocks_per_sm(stencil2d_kernel<T, false>, kThreads2);
+    const long long slots = slots4 * kWarps2 / wpb;
     if (small_problem(a.height, per_band, 8, slots)) band_h = pick_band_height_small(a.height, per_band, 2 * T + 1, 8, 128, slots);
-    dim3 grid((strips + kWarps2 - 1) / kWarps2, (a.height + band_h - 1) / band_h, a.batch);
+    dim3 grid((strips + wpb - 1) / wpb, (a.height + band_h - 1) / band_h, a.batch);
     if (grid.y > 65535 || a.batch > 65535) return cudaErrorInvalidConfiguration;
-    if (five) launch_kernel(stencil2d_kernel<T, true>, grid, kThreads2, s, a, coef, band_h);
-    else launch_kernel(stencil2d_kernel<T, false>, grid, kThreads2, s, a, coef, band_h);
+    if (five) launch_kernel(stencil2d_kernel<T, true>, grid, wpb * kLanes, s, a, coef, band_h);
+    else launch_kernel(stencil2d_kernel<T, false>, grid, wpb * kLanes, s, a, coef, band_h);
     return cudaGetLastError();
 }
 
