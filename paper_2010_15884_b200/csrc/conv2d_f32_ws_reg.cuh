@@ -1,10 +1,10 @@
-// 2-D fp32 weight-stationary convolution for the smaller filters (at most 8 filter columns, window of at most 96
-// registers: up to 9 x 8 and 15 x 4): the arrays
+// 2-D fp32 weight-stationary convolution for the smaller filters (at most 8 filter columns and a window of at most
+// 96 registers: up to 9 x 8 and 15 x 4; wider filters of one or two rows): the arrays
 // side by side ALONG THE ROWS, everything in registers, no shared memory.
 //
 // As in the other weight-stationary kernels an array (Q PEs, PE q keeps the P taps of filter column q) is folded
 // into one lane, the taps are uniform operands and the sums of two neighbouring outputs travel as a register
-// pair updated by one packed fp32x2 FMA per tap.  Here array a (lane a) takes the SEG = 4 or 8 image columns
+// pair updated by one packed fp32x2 FMA per tap.  Here array a (lane a) takes the SEG = 4, 8 or 16 image columns
 // [c0 + SEG*a, c0 + SEG*(a+1)) of a row group: exactly the columns its lane fetches with its own 128-bit loads,
 // which are contiguous across the warp -- the broadcast input of macro-step T is simply register T of that load,
 // so no transpose and no staging is needed.  Every array runs exactly SEG macro-steps, neither filling nor
@@ -28,10 +28,12 @@ constexpr int kWsrWarps = 4;
 
 template <int P, int Q>
 struct WsrShape {
-    static constexpr int kSeg = Q <= 4 ? 4 : 8;                 // image columns per array and pass
+    static constexpr int kSeg = Q <= 4 ? 4 : Q <= 8 ? 8 : 16;   // image columns per array and pass
     // window registers: (P+3) x segment.  Measured on 2 x 2048 x 4096 against the form with transposed staging: 6x5
     // 65 -> 37 us, 7x7 72 -> 50, 8x6 73 -> 52, 9x7 79 -> 70, 9x8 level; 11 rows: 11x5 76 -> 66 but 11x8 86 -> 104
-    static constexpr bool kFits = Q <= 8 && (P + kWsrM - 1) * kSeg <= 96;
+    // 16-column segments (filters of 9 to 15 columns) pay for one and two filter rows (1x15 52 -> 38 us, 2x13 66 -> 45);
+    // with three rows the two forms are level
+    static constexpr bool kFits = kSeg == 16 ? P <= 2 : (P + kWsrM - 1) * kSeg <= 96;
     static constexpr int kOut = (kLanes - 1) * kSeg;            // output columns per warp
 };
 

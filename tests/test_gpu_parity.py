@@ -530,7 +530,8 @@ BAD_PIXELS = ((0, 0, np.inf), (40, 127, np.nan), (41, 128, -np.inf), (63, 255, n
               (119, 299, np.inf), (100, 5, np.inf))
 
 
-@pytest.mark.parametrize("pq", [(6, 5), (7, 8), (8, 7), (9, 8), (9, 5), (15, 4), (14, 3), (11, 4), (13, 2)],
+@pytest.mark.parametrize("pq", [(6, 5), (7, 8), (8, 7), (9, 8), (9, 5), (15, 4), (14, 3), (11, 4), (13, 2), (1, 9), (1, 15), (2, 12),
+                                (2, 15), (1, 14)],
                          ids=lambda f: "%dx%d" % f)
 def test_2d_ws_register_form_taller_filters(cuda_device, pq):
     """The all-register weight-stationary form takes every filter of at most 8 columns whose window of P+3 rows fits
