@@ -13,26 +13,26 @@
 // Arrays neither fill nor drain: each runs exactly the 16 macro-steps of its segment.  The sums of the last
 // 4*(G-1) outputs of a segment are completed by the next array, which starts from empty PEs and hands its share
 // back by shuffle (integer addition is exact in any order).  Lane 31 is only such a successor: a warp yields
-// 31 * 16 output columns.  Four output rows are computed per pass; every input row of the pass is fetched once,
-// its 16 shifted words are built once and used by up to four output rows.
+// 31 * 16 output columns.  Four output rows (two for filters of up to four rows) are computed per pass; every input
+// row of the pass is fetched once, its 16 shifted words are built once and used by up to four output rows.
 #pragma once
 
 #include "conv2d_u8_dp4a.cuh"
 
 namespace sysconv {
 
-constexpr int kU8WsM = 4;                       // output rows per pass
+constexpr int kU8WsM = 4;                       // output rows per pass (two for filters of up to four rows)
 constexpr int kU8WsWarps = 4;
 constexpr int kU8WsSeg = 16;                    // pixels per array and pass (one 128-bit load)
 constexpr int kU8WsOut = (kLanes - 1) * kU8WsSeg;
 constexpr int kU8WsPitch = kU8WsSeg + 4;        // ints per lane block of the output staging row
 
-template <int P, int Q>
+template <int P, int Q, int MROWS = kU8WsM>
 __global__ void __launch_bounds__(kU8WsWarps *kLanes)
 conv2d_u8_ws_dp4a_kernel(const Conv2DArgs a, const __grid_constant__ TapsPacked taps, const int band_h)
 {
     dependent_launch_enter();
-    constexpr int M = kU8WsM, K = M + P - 1, G = (Q + 3) / 4, SEG = kU8WsSeg, TAIL = 4 * (G - 1);
+    constexpr int M = MROWS, K = M + P - 1, G = (Q + 3) / 4, SEG = kU8WsSeg, TAIL = 4 * (G - 1);
     const int lane = threadIdx.x & (kLanes - 1);
     const int slice = blockIdx.x * kU8WsWarps + threadIdx.x / kLanes;    // (a block of fewer warps is the only one of its row)
     const int c0 = slice * kU8WsOut;                    // first output column of the slice
@@ -170,8 +170,8 @@ inline bool u8_ws_dp4a_eligible(const Conv2DArgs &a)
     return (xa & 15ull) == 0 && (a.x_pitch & 15) == 0 && (a.batch == 1 || (a.x_bstride & 15) == 0);
 }
 
-template <int P, int Q>
-cudaError_t launch_conv2d_u8_ws_dp4a(const Conv2DArgs &a, const Taps2DInt &t, cudaStream_t s)
+template <int P, int Q, int MROWS>
+cudaError_t launch_conv2d_u8_ws_dp4a_m(const Conv2DArgs &a, const Taps2DInt &t, cudaStream_t s)
 {
     TapsPacked pk;
     for (int p = 0; p < kMaxP2; ++p)
@@ -187,21 +187,30 @@ cudaError_t launch_conv2d_u8_ws_dp4a(const Conv2DArgs &a, const Taps2DInt &t, cu
     const int slices = (a.out_w + kU8WsOut - 1) / kU8WsOut;
     const int wpb = block_warps(slices, kU8WsWarps);
     const long long per_band = static_cast<long long>((slices + wpb - 1) / wpb) * a.batch;
-    static const long long slots4 = 148LL * resident_blocks_per_sm(conv2d_u8_ws_dp4a_kernel<P, Q>, kU8WsWarps * kLanes);
+    static const long long slots4 = 148LL * resident_blocks_per_sm(conv2d_u8_ws_dp4a_kernel<P, Q, MROWS>, kU8WsWarps * kLanes);
     const long long slots = slots4 * kU8WsWarps / wpb;      // smaller blocks: as many more of them are resident
     long long band_h;
-    if (small_problem(a.out_h, per_band, kU8WsM, slots)) {
-        band_h = pick_band_height_small(a.out_h, per_band, P, kU8WsM, 64, slots);
+    if (small_problem(a.out_h, per_band, MROWS, slots)) {
+        band_h = pick_band_height_small(a.out_h, per_band, P, MROWS, 64, slots);
     } else {
         const long long bands = (148LL * 16 + per_band - 1) / per_band;
         band_h = (a.out_h + bands - 1) / bands;
         if (band_h > 64) band_h = 64;
     }
-    band_h = (band_h + kU8WsM - 1) / kU8WsM * kU8WsM;
-    if ((a.out_h + band_h - 1) / band_h > 65535) band_h = ((a.out_h + 65534) / 65535 + kU8WsM - 1) / kU8WsM * kU8WsM;
+    band_h = (band_h + MROWS - 1) / MROWS * MROWS;
+    if ((a.out_h + band_h - 1) / band_h > 65535) band_h = ((a.out_h + 65534) / 65535 + MROWS - 1) / MROWS * MROWS;
     dim3 grid((slices + wpb - 1) / wpb, static_cast<unsigned>((a.out_h + band_h - 1) / band_h), a.batch);
-    launch_kernel(conv2d_u8_ws_dp4a_kernel<P, Q>, grid, wpb * kLanes, s, a, pk, static_cast<int>(band_h));
+    launch_kernel(conv2d_u8_ws_dp4a_kernel<P, Q, MROWS>, grid, wpb * kLanes, s, a, pk, static_cast<int>(band_h));
     return cudaGetLastError();
+}
+
+template <int P, int Q>
+cudaError_t launch_conv2d_u8_ws_dp4a(const Conv2DArgs &a, const Taps2DInt &t, cudaStream_t s)
+{
+    // up to four filter rows: two output rows per pass (half the accumulators, more blocks per SM; 3840 x 2160, 3x3:
+    // 15.9 -> 14.1 us); taller filters: four, so that an input row serves up to four output rows
+    if constexpr (P <= 4) return launch_conv2d_u8_ws_dp4a_m<P, Q, 2>(a, t, s);
+    else return launch_conv2d_u8_ws_dp4a_m<P, Q, kU8WsM>(a, t, s);
 }
 
 // uint8 rows that start 16-byte aligned run on the packed weight-stationary kernel
